@@ -1,0 +1,170 @@
+/*
+ * kvc -- budgeted KV cache for block-wise ("compress as you prefill") multimodal prefill on B200.
+ *
+ * C ABI.  No exception crosses it; every function returns an int status (0 = KVC_OK) unless noted.
+ * All tensor arguments are raw pointers; whether a pointer is HOST or DEVICE memory is stated per
+ * argument.  The caller owns every device buffer (cache blobs, workspace, q/k/v/out); the context
+ * owns only host-side state (configuration and the current cache length of every layer).
+ *
+ * The library implements the per-block body of the paper's Alg. 1 ("Block-wise Prefill with KV
+ * Eviction"): the caller loops over blocks (and layers) and calls kvc_prefill_chunk once per
+ * (block, layer).  Notation: L layers, Hq query heads, Hkv kv-heads, G = Hq/Hkv, d = head_dim,
+ * B = budget (the paper's M), n = tokens in this block (the paper's b), n_c = cache length before
+ * the call, tot = n_c + n, w = observer window, cap = B + max_chunk rounded up to 128.
+ *
+ * One call does, on the caller's stream, for every kv-head independently:
+ *   a0  append   C <- C u (K_i, V_i)                                          (Alg. 1)
+ *   a1  attend   out = softmax(q k^T / sqrt(d)) v over cache u block, causal
+ *                inside the block                                             (Eq. 1)
+ *   a2  score    if tot > B: importance of every cached key = attention probability it receives
+ *                from the observer queries (the block's last w rows), summed over those rows and
+ *                over the G query heads sharing the kv-head                   (Eq. 4)
+ *   a3  select   evict the tot - B lowest-scoring entries; ties keep the older entry; the
+ *                observers' own w keys are never evicted                      (Alg. 1, Evict)
+ *   a4  compact  retained entries are moved into rows [0, B); length becomes B (Sec. 3.1)
+ */
+#ifndef KVC_H_
+#define KVC_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvc_ctx kvc_ctx; /* opaque, host memory, created/destroyed by the library */
+
+/* status codes */
+#define KVC_OK        0
+#define KVC_EINVAL   -1  /* bad configuration or argument (null/misaligned pointer, n out of range, ...) */
+#define KVC_ESTATE   -2  /* call order violated (layer not reset, destroyed context, ...)              */
+#define KVC_ECUDA    -3  /* a CUDA call or launch failed; text in kvc_last_error                       */
+#define KVC_ETIMEOUT -4  /* a bounded device-side wait ran out (reported by kvc_status)                */
+
+typedef enum { KVC_F32 = 0, KVC_BF16 = 1 } kvc_dtype;
+typedef enum { KVC_SCORE_ATTN = 0 /* query-aware score, Eq. 4 */ } kvc_policy;
+
+/* flags */
+#define KVC_FLAG_CUDA_CORES 1u /* bf16 only: run attention/score on the CUDA-core kernels used for
+                                  fp32 instead of the tcgen05 tensor-core kernels (diagnostic) */
+
+typedef struct {
+  int n_layers;        /* L >= 1                                                                 */
+  int n_q_heads;       /* Hq, multiple of n_kv_heads; consecutive query heads share a kv-head     */
+  int n_kv_heads;      /* Hkv                                                                     */
+  int head_dim;        /* d in {64, 128}                                                          */
+  int dtype;           /* kvc_dtype of q/k/v/out and of the cached keys/values                    */
+  int budget;          /* B: entries kept per (layer, kv-head) = memory budget M of Alg. 1        */
+  int max_chunk;       /* largest n ever passed = block size b of Alg. 1                          */
+  int obs_window;      /* w; 0 -> 32.  The window used by a call is min(w, n); needs w <= B       */
+  int policy;          /* kvc_policy                                                              */
+  float softmax_scale; /* 0 -> 1/sqrt(head_dim) as in Eq. 1 and Eq. 4                             */
+  int device;          /* CUDA device ordinal the context is bound to                             */
+  unsigned flags;      /* KVC_FLAG_*                                                              */
+} kvc_config;
+
+/* Borrowed view of one layer's cache (pointers into the caller's cache blob, nothing is copied).
+ * Rows [len, cap) are unspecified.  The order of entries is unspecified; pos identifies them. */
+typedef struct {
+  void* k;              /* DEVICE  [Hkv][cap][d], dtype                      */
+  void* v;              /* DEVICE  [Hkv][cap][d], dtype                      */
+  int* pos;             /* DEVICE  [Hkv][cap] int32, absolute token position */
+  int len;              /* valid entries per kv-head (same for every head)   */
+  int cap;              /* row capacity per kv-head                          */
+  int n_kv_heads, head_dim, dtype;
+} kvc_view;
+
+/* Sec. 3, Alg. 1 inputs (block size b, budget M) plus the attention shape.  Validates the
+ * configuration (Hq % Hkv == 0, d in {64,128}, 1 <= w <= B, max_chunk >= 1, G <= 128) and creates
+ * the host context.  *out is set to NULL on failure.  Allocates no device memory. */
+int kvc_create(const kvc_config* cfg, kvc_ctx** out);
+
+/* Frees the host context.  Device buffers stay with the caller. */
+int kvc_destroy(kvc_ctx* ctx);
+
+/* Sizes the caller must allocate (device memory, 256-byte aligned): per_layer = bytes of one
+ * layer's cache blob (K, V, pos; this is the physical bound of Eq. 2 with sequence length cap);
+ * workspace = bytes of the scratch area shared by all layers (log-sum-exp of the last block,
+ * scores, move lists, status word).  Either pointer may be NULL. */
+int kvc_cache_nbytes(const kvc_ctx* ctx, size_t* per_layer, size_t* workspace);
+
+/* Clears the workspace header (status word).  Call once after allocating a workspace, before the
+ * first kvc_prefill_chunk that uses it.  Asynchronous on `stream`. */
+int kvc_workspace_init(kvc_ctx* ctx, void* workspace, void* stream);
+
+/* Alg. 1 "C <- empty" for `n_layers` consecutive layers starting at `layer`: zero-fills the blobs
+ * (asynchronously on `stream`) and sets their length to 0.  Must precede the first
+ * kvc_prefill_chunk of a layer.  cache: DEVICE, blob of layer `layer`; blobs of consecutive
+ * layers are cache_layer_stride bytes apart (ignored when n_layers == 1). */
+int kvc_reset(kvc_ctx* ctx, int layer, int n_layers, void* cache, size_t cache_layer_stride,
+              void* stream);
+
+/* The body of Alg. 1's loop for one block and one layer (steps a0..a4 above; Eq. 1, Eq. 4).
+ *   q   DEVICE [n][Hq ][d]  queries of the block (already position-encoded), dtype
+ *   k,v DEVICE [n][Hkv][d]  keys / values of the block, dtype
+ *   n   1 <= n <= max_chunk; pos0 = absolute position of the block's first token
+ *   cache      DEVICE this layer's blob (kvc_cache_nbytes per_layer bytes); read and written
+ *   workspace  DEVICE scratch (kvc_cache_nbytes workspace bytes); calls sharing a workspace must
+ *              be ordered on one stream
+ *   out DEVICE [n][Hq][d]   attention output, dtype
+ *   stream     cudaStream_t; the call only enqueues work and returns
+ * All pointers must be 16-byte aligned.  Returns KVC_EINVAL / KVC_ESTATE / KVC_ECUDA without
+ * enqueuing anything on failure of the host checks. */
+int kvc_prefill_chunk(kvc_ctx* ctx, int layer, const void* q, const void* k, const void* v, int n,
+                      long long pos0, void* cache, void* workspace, void* out, void* stream);
+
+/* Same as kvc_prefill_chunk for `n_layers` consecutive layers in one set of launches (the layer
+ * index becomes a grid dimension).  Only meaningful when every layer's q/k/v exist up front
+ * (synthetic inputs, or layers of independent models); a real decoder stack cannot use it because
+ * layer l+1's input depends on layer l's output.  Layer i's tensors are at q + i*q_layer_stride
+ * (strides in ELEMENTS for q/k/v/out, in BYTES for the cache).  All layers must hold the same
+ * cache length. */
+int kvc_prefill_chunk_layers(kvc_ctx* ctx, int layer0, int n_layers, const void* q,
+                             long long q_layer_stride, const void* k, const void* v,
+                             long long kv_layer_stride, int n, long long pos0, void* cache,
+                             size_t cache_layer_stride, void* workspace, void* out,
+                             long long out_layer_stride, void* stream);
+
+/* Bytes of the DEVICE staging buffer kvc_prefill_chunk_host needs (room for q, k, v and out of a
+ * block of max_chunk tokens). */
+int kvc_staging_nbytes(const kvc_ctx* ctx, size_t* nbytes);
+
+/* kvc_prefill_chunk with HOST q/k/v/out (pinned memory recommended): copies the block's q, k, v
+ * into `staging` (DEVICE, kvc_staging_nbytes bytes, 256-byte aligned), runs the block, copies `out`
+ * back to the host.  Everything is asynchronous on `stream`; out_host is valid after the stream
+ * is synchronised. */
+int kvc_prefill_chunk_host(kvc_ctx* ctx, int layer, const void* q_host, const void* k_host,
+                           const void* v_host, int n, long long pos0, void* cache, void* workspace,
+                           void* staging, void* out_host, void* stream);
+
+/* Output of Alg. 1: the compressed cache of one layer, as borrowed pointers. */
+int kvc_cache_view(const kvc_ctx* ctx, int layer, void* cache, kvc_view* view);
+
+/* Pointers into the workspace for inspection after a call (DEVICE, borrowed):
+ *   lse    [n][Hq] fp32   natural-log log-sum-exp of every row's scaled scores (Eq. 1 normaliser)
+ *   score  [Hkv][cap] fp32 importance of entry j before compaction (Eq. 4), valid for j < tot - w
+ * of the most recent call for layer slot `slot` (0 for single-layer calls, i for layer layer0+i of
+ * a batched call). */
+int kvc_workspace_view(const kvc_ctx* ctx, void* workspace, int slot, float** lse, float** score);
+
+/* Synchronises `stream` and returns the device status word kept in the workspace: KVC_OK, or
+ * KVC_ETIMEOUT if a bounded wait inside a kernel gave up (the kernel then left early; results of
+ * that call are invalid but the context and the device stay usable). */
+int kvc_status(kvc_ctx* ctx, void* workspace, void* stream);
+
+/* KV bytes after Eq. 2 (2 x layers x heads x dim_head x precision x sequence length):
+ * logical uses sequence length B, physical uses cap (what the blobs really hold, pos excluded),
+ * uncompressed uses seq_len. */
+int kvc_kv_bytes(const kvc_ctx* ctx, long long seq_len, size_t* logical, size_t* physical,
+                 size_t* uncompressed);
+
+/* Number of kernel launches the library has enqueued through this context so far. */
+long long kvc_launch_count(const kvc_ctx* ctx);
+
+/* Text of the most recent error of this context (never NULL; valid until the next call). */
+const char* kvc_last_error(const kvc_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVC_H_ */

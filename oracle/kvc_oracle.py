@@ -96,7 +96,9 @@ class KVCOracle:
         self.pos[layer][g], self.K[layer][g], self.V[layer][g] = allpos[idx], allK[idx], allV[idx]
 
     # ------------------------------------------------------------------------------------
-    def prefill_chunk(self, layer: int, q, k, v, pos0: int) -> ChunkResult:
+    def prefill_chunk(self, layer: int, q, k, v, pos0: int, kv_heads=None) -> ChunkResult:
+        """One block of Alg. 1 for one layer.  ``kv_heads`` restricts the work to a subset of kv-heads
+        (they are independent); the other heads' state and outputs are left untouched (zeros)."""
         q = np.asarray(q, dtype=np.float64)
         k = np.asarray(k, dtype=np.float64)
         v = np.asarray(v, dtype=np.float64)
@@ -111,6 +113,9 @@ class KVCOracle:
             self._pre_evict = [[None] * self.Hkv for _ in range(self.L)]
 
         for g in range(self.Hkv):
+            if kv_heads is not None and g not in kv_heads:
+                scores.append(None); cand_pos.append(None); gaps.append(None); retained.append(None)
+                continue
             # 1. append (Alg. 1): the block's keys/values join the cache before anything is evicted
             n_c = len(self.pos[layer][g])
             pos = np.concatenate([self.pos[layer][g], pos0 + np.arange(n, dtype=np.int64)])

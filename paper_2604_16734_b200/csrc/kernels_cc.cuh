@@ -1,0 +1,351 @@
+// CUDA-core kernels: append (a0), fp32-accurate attention (a1) and score (a2) for fp32 inputs
+// (and, as a diagnostic, bf16 inputs), exact per-head selection (a3) and hole-fill compaction (a4).
+#pragma once
+#include "geom.cuh"
+
+namespace kvc {
+
+// ------------------------------------------------------------------------------------------------
+// a0 append (Alg. 1: C <- C u (K_i, V_i)).  One warp per (token, kv-head) row: copies the K and V
+// rows into cache rows n_c + t and records the absolute position.
+// grid (ceil(n*Hkv / 8), 1, nl), block 256.
+template <typename T>
+__global__ void __launch_bounds__(256) append_kernel(const T* __restrict__ k, const T* __restrict__ v,
+                                                     char* __restrict__ cache, Geom p) {
+  const int layer = blockIdx.z;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= p.n * p.Hkv) return;
+  const int t = row / p.Hkv, g = row % p.Hkv;
+  char* blob = cache + layer * p.cache_ls;
+  const int vec_per_row = p.d * (int)sizeof(T) / 16;
+  const uint4* ksrc = reinterpret_cast<const uint4*>(k + layer * p.kv_ls + (static_cast<long long>(t) * p.Hkv + g) * p.d);
+  const uint4* vsrc = reinterpret_cast<const uint4*>(v + layer * p.kv_ls + (static_cast<long long>(t) * p.Hkv + g) * p.d);
+  const long long dst_row = static_cast<long long>(g) * p.cap + p.n_c + t;
+  uint4* kdst = reinterpret_cast<uint4*>(blob + dst_row * p.d * sizeof(T));
+  uint4* vdst = reinterpret_cast<uint4*>(blob + p.v_off + dst_row * p.d * sizeof(T));
+  for (int i = lane; i < vec_per_row; i += 32) {
+    kdst[i] = ksrc[i];
+    vdst[i] = vsrc[i];
+  }
+  if (lane == 0) reinterpret_cast<int*>(blob + p.pos_off)[dst_row] = static_cast<int>(p.pos0 + t);
+}
+
+// ------------------------------------------------------------------------------------------------
+// a1 attention on CUDA cores (Eq. 1), fp32 arithmetic throughout.
+// Block = 4 warps x 4 rows = 16 tokens of one query head; keys/values stream through shared memory
+// 32 at a time.  In the score phase lane j owns key j of the tile; in the PV phase lane c owns
+// output columns c, c+32, ....  grid (ceil(n/16), Hq, nl), block 128.
+template <typename T, int D>
+__global__ void __launch_bounds__(128) attn_cc_kernel(const T* __restrict__ q, const char* __restrict__ cache,
+                                                      T* __restrict__ out, char* __restrict__ ws, Geom p) {
+  constexpr int RW = 4, KT = 32, KS = D + 4, NC = D / 32;
+  __shared__ __align__(16) float sK[KT * KS];
+  __shared__ __align__(16) float sV[KT * D];
+  __shared__ __align__(16) float sQ[16 * D];
+  const int layer = blockIdx.z, h = blockIdx.y, g = h / p.G;
+  const int tok0 = blockIdx.x * 16;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const char* blob = cache + layer * p.cache_ls;
+  const T* Kc = reinterpret_cast<const T*>(blob) + static_cast<long long>(g) * p.cap * D;
+  const T* Vc = reinterpret_cast<const T*>(blob + p.v_off) + static_cast<long long>(g) * p.cap * D;
+  const T* qb = q + layer * p.q_ls;
+
+  for (int i = threadIdx.x; i < 16 * D; i += 128) {
+    const int r = i / D, c = i % D, tok = tok0 + r;
+    sQ[i] = tok < p.n ? to_f32<T>(qb[(static_cast<long long>(tok) * p.Hq + h) * D + c]) : 0.f;
+  }
+
+  float m[RW], l[RW], acc[RW][NC];
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    m[r] = -INFINITY; l[r] = 0.f;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) acc[r][c] = 0.f;
+  }
+  const int last_tok = min(tok0 + 16, p.n) - 1;
+  const int kv_end = p.n_c + last_tok + 1;          // keys visible to the last row of this block
+
+  for (int t0 = 0; t0 < kv_end; t0 += KT) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < KT * D; i += 128) {
+      const int j = i / D, c = i % D, key = t0 + j;
+      float kk = 0.f, vv = 0.f;
+      if (key < kv_end) {
+        kk = to_f32<T>(Kc[static_cast<long long>(key) * D + c]);
+        vv = to_f32<T>(Vc[static_cast<long long>(key) * D + c]);
+      }
+      sK[j * KS + c] = kk;
+      sV[j * D + c] = vv;
+    }
+    __syncthreads();
+
+    float s[RW];
+#pragma unroll
+    for (int r = 0; r < RW; ++r) s[r] = 0.f;
+    const float4* krow = reinterpret_cast<const float4*>(&sK[lane * KS]);
+#pragma unroll 8
+    for (int c4 = 0; c4 < D / 4; ++c4) {
+      const float4 kv = krow[c4];
+#pragma unroll
+      for (int r = 0; r < RW; ++r) {
+        const float4 qv = reinterpret_cast<const float4*>(&sQ[(warp * RW + r) * D])[c4];
+        s[r] = fmaf(qv.x, kv.x, s[r]); s[r] = fmaf(qv.y, kv.y, s[r]);
+        s[r] = fmaf(qv.z, kv.z, s[r]); s[r] = fmaf(qv.w, kv.w, s[r]);
+      }
+    }
+    const int key = t0 + lane;
+    float pr[RW];
+#pragma unroll
+    for (int r = 0; r < RW; ++r) {
+      const int tok = tok0 + warp * RW + r;
+      const bool vis = tok < p.n && key < p.n_c + tok + 1;     // causal inside the block only
+      const float t = vis ? s[r] * p.scale_log2 : -INFINITY;
+      float tmax = t;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+      const float m_new = fmaxf(m[r], tmax);
+      float pv = 0.f, corr = 1.f;
+      if (m_new != -INFINITY) {
+        pv = exp2f(t - m_new);
+        corr = exp2f(m[r] - m_new);
+      }
+      float psum = pv;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, o);
+      l[r] = l[r] * corr + psum;
+      m[r] = m_new;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) acc[r][c] *= corr;
+      pr[r] = pv;
+    }
+#pragma unroll 4
+    for (int j = 0; j < KT; ++j) {
+      float vj[NC];
+#pragma unroll
+      for (int c = 0; c < NC; ++c) vj[c] = sV[j * D + lane + 32 * c];
+#pragma unroll
+      for (int r = 0; r < RW; ++r) {
+        const float pj = __shfl_sync(0xffffffffu, pr[r], j);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) acc[r][c] = fmaf(pj, vj[c], acc[r][c]);
+      }
+    }
+  }
+
+  float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
+  T* ob = out + layer * p.out_ls;
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    const int tok = tok0 + warp * RW + r;
+    if (tok >= p.n) continue;
+    const float inv = 1.f / l[r];
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+      ob[(static_cast<long long>(tok) * p.Hq + h) * D + lane + 32 * c] = from_f32<T>(acc[r][c] * inv);
+    if (lane == 0) lse[static_cast<long long>(tok) * p.Hq + h] = (m[r] + log2f(l[r])) * 0.6931471805599453f;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// a2 score on CUDA cores (Eq. 4): score_j = sum over the w observer rows and the G heads of the
+// group of 2^(s_ij*scale_log2 - lse2_i).  Thread t owns candidate key blockIdx.x*128 + t.
+// grid (ceil(n_cand/128), Hkv, nl), block 128, dynamic smem = 128*(D+4)*4 + 32*D*4 + 32*4 bytes.
+template <typename T, int D>
+__global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, const char* __restrict__ cache,
+                                                       char* __restrict__ ws, Geom p) {
+  constexpr int KS = D + 4;
+  extern __shared__ __align__(16) float smem_f[];
+  float* sK = smem_f;                 // [128][KS]
+  float* sQ = sK + 128 * KS;          // [32][D]
+  float* sL = sQ + 32 * D;            // [32]
+  const int layer = blockIdx.z, g = blockIdx.y;
+  const int key0 = blockIdx.x * 128;
+  const char* blob = cache + layer * p.cache_ls;
+  const T* Kc = reinterpret_cast<const T*>(blob) + static_cast<long long>(g) * p.cap * D;
+  const T* qb = q + layer * p.q_ls;
+  char* slot = ws_slot(ws, p, layer);
+  const float* lse = reinterpret_cast<const float*>(slot + p.lse_off);
+  float* score = reinterpret_cast<float*>(slot + p.score_off) + static_cast<long long>(g) * p.cap;
+
+  for (int i = threadIdx.x; i < 128 * D; i += 128) {
+    const int j = i / D, c = i % D, key = key0 + j;
+    sK[j * KS + c] = key < p.n_cand ? to_f32<T>(Kc[static_cast<long long>(key) * D + c]) : 0.f;
+  }
+  const int rows = p.w * p.G;
+  float acc = 0.f;
+  const float4* krow = reinterpret_cast<const float4*>(&sK[threadIdx.x * KS]);
+  for (int r0 = 0; r0 < rows; r0 += 32) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < 32 * D; i += 128) {
+      const int r = r0 + i / D, c = i % D;
+      float x = 0.f;
+      if (r < rows) {
+        const int tok = p.n - p.w + r / p.G, h = g * p.G + r % p.G;
+        x = to_f32<T>(qb[(static_cast<long long>(tok) * p.Hq + h) * D + c]);
+      }
+      sQ[i] = x;
+    }
+    if (threadIdx.x < 32) {
+      const int r = r0 + threadIdx.x;
+      float lv = INFINITY;                                   // padding rows contribute 2^-inf = 0
+      if (r < rows) {
+        const int tok = p.n - p.w + r / p.G, h = g * p.G + r % p.G;
+        lv = lse[static_cast<long long>(tok) * p.Hq + h] * 1.4426950408889634f;
+      }
+      sL[threadIdx.x] = lv;
+    }
+    __syncthreads();
+    const int rmax = min(32, rows - r0);
+    for (int r = 0; r < rmax; ++r) {
+      const float4* qrow = reinterpret_cast<const float4*>(&sQ[r * D]);
+      float s = 0.f;
+#pragma unroll 8
+      for (int c4 = 0; c4 < D / 4; ++c4) {
+        const float4 a = qrow[c4], b = krow[c4];
+        s = fmaf(a.x, b.x, s); s = fmaf(a.y, b.y, s); s = fmaf(a.z, b.z, s); s = fmaf(a.w, b.w, s);
+      }
+      acc += exp2f(s * p.scale_log2 - sL[r]);
+    }
+  }
+  const int key = key0 + threadIdx.x;
+  if (key < p.n_cand) score[key] = acc;
+}
+
+// ------------------------------------------------------------------------------------------------
+// a3 select (Alg. 1 Evict): one CTA per (kv-head, layer).  Exact radix select of the n_keep-th
+// largest 64-bit key (score bits high, inverted position low: larger key = higher score, then
+// older entry), then ordered lists of the holes below B and of the survivors at or above B.
+// Scores are sums of probabilities, hence >= 0, so their IEEE bit patterns order like integers.
+// grid (Hkv, 1, nl), block 1024.
+__device__ __forceinline__ unsigned long long select_key(float score, int pos) {
+  return (static_cast<unsigned long long>(__float_as_uint(score)) << 32) |
+         static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(pos));
+}
+
+__global__ void __launch_bounds__(1024) select_kernel(const char* __restrict__ cache, char* __restrict__ ws, Geom p) {
+  __shared__ int hist[256];
+  __shared__ int warp_tot[32];
+  __shared__ unsigned long long s_prefix;
+  __shared__ int s_remaining;
+  __shared__ int s_base;
+  const int layer = blockIdx.z, g = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const char* blob = cache + layer * p.cache_ls;
+  const int* pos = reinterpret_cast<const int*>(blob + p.pos_off) + static_cast<long long>(g) * p.cap;
+  char* slot = ws_slot(ws, p, layer);
+  const float* score = reinterpret_cast<const float*>(slot + p.score_off) + static_cast<long long>(g) * p.cap;
+  int* msrc = reinterpret_cast<int*>(slot + p.msrc_off) + static_cast<long long>(g) * p.max_chunk;
+  int* mdst = reinterpret_cast<int*>(slot + p.mdst_off) + static_cast<long long>(g) * p.max_chunk;
+  int* mcount = reinterpret_cast<int*>(slot + p.mcount_off);
+
+  // ---- threshold: the n_keep-th largest key among the n_cand candidates (n_keep >= 1 here)
+  unsigned long long thr = ~0ull;            // n_keep == 0: nothing among the candidates survives
+  if (p.n_keep > 0) {
+    if (tid == 0) { s_prefix = 0ull; s_remaining = p.n_keep; }
+    for (int shift = 56; shift >= 0; shift -= 8) {
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      const unsigned long long prefix = s_prefix;
+      const int remaining = s_remaining;
+      for (int j = tid; j < p.n_cand; j += 1024) {
+        const unsigned long long key = select_key(score[j], pos[j]);
+        const bool match = (shift == 56) || ((key >> (shift + 8)) == (prefix >> (shift + 8)));
+        if (match) atomicAdd(&hist[(key >> shift) & 255], 1);
+      }
+      __syncthreads();
+      // descending scan over bins: thread t looks at bin 255 - t
+      int cnt = 0, incl = 0;
+      if (tid < 256) {
+        cnt = hist[255 - tid];
+        incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += y;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+      }
+      __syncthreads();
+      if (tid < 256) {
+        int off = 0;
+        for (int wq = 0; wq < warp; ++wq) off += warp_tot[wq];
+        incl += off;
+        if (incl >= remaining && incl - cnt < remaining) {     // exactly one bin satisfies this
+          s_prefix = prefix | (static_cast<unsigned long long>(255 - tid) << shift);
+          s_remaining = remaining - (incl - cnt);
+        }
+      }
+      __syncthreads();
+    }
+    thr = s_prefix;
+  }
+
+  // ---- holes: evicted entries in rows [0, B); survivors: retained entries in rows [B, tot).
+  // Entry j is retained iff it is protected (j >= n_cand) or its key >= thr.  Both lists are
+  // produced in ascending row order (block-wide exclusive scans over contiguous segments).
+  for (int pass = 0; pass < 2; ++pass) {
+    const int lo = pass == 0 ? 0 : p.B;
+    const int hi = pass == 0 ? min(p.B, p.tot) : p.tot;
+    const int per = (hi - lo + 1023) / 1024;
+    const int j0 = lo + tid * per, j1 = min(j0 + per, hi);
+    int cnt = 0;
+    for (int j = j0; j < j1; ++j) {
+      const bool kept = j >= p.n_cand || (p.n_keep > 0 && select_key(score[j], pos[j]) >= thr);
+      cnt += (pass == 0) ? !kept : kept;
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    __syncthreads();
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int off = 0;
+    for (int wq = 0; wq < warp; ++wq) off += warp_tot[wq];
+    int rank = off + incl - cnt;
+    int* list = pass == 0 ? mdst : msrc;
+    for (int j = j0; j < j1; ++j) {
+      const bool kept = j >= p.n_cand || (p.n_keep > 0 && select_key(score[j], pos[j]) >= thr);
+      if ((pass == 0) ? !kept : kept) list[rank++] = j;
+    }
+    if (pass == 0 && tid == 1023) s_base = off + incl;       // number of holes = number of moves
+    __syncthreads();
+  }
+  if (tid == 0) mcount[g] = s_base;
+}
+
+// ------------------------------------------------------------------------------------------------
+// a4 compact: move m copies the K row, the V row and the position of entry src[m] (>= B) into the
+// hole dst[m] (< B).  Sources and destinations never overlap, rows are copied bit-exactly.
+// One warp per move.  grid (ceil(max_moves/8), Hkv, nl), block 256.
+__global__ void __launch_bounds__(256) compact_kernel(char* __restrict__ cache, const char* __restrict__ ws, Geom p,
+                                                      int elem_bytes) {
+  const int layer = blockIdx.z, g = blockIdx.y;
+  const int mv = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  const char* slot = ws + kWsHeaderBytes + static_cast<long long>(layer) * p.ws_ls;
+  const int count = reinterpret_cast<const int*>(slot + p.mcount_off)[g];
+  if (mv >= count) return;
+  const int src = reinterpret_cast<const int*>(slot + p.msrc_off)[static_cast<long long>(g) * p.max_chunk + mv];
+  const int dst = reinterpret_cast<const int*>(slot + p.mdst_off)[static_cast<long long>(g) * p.max_chunk + mv];
+  char* blob = cache + layer * p.cache_ls;
+  const long long row_bytes = static_cast<long long>(p.d) * elem_bytes;
+  const int vec = static_cast<int>(row_bytes / 16);
+  const long long head = static_cast<long long>(g) * p.cap;
+  const uint4* ks = reinterpret_cast<const uint4*>(blob + (head + src) * row_bytes);
+  const uint4* vs = reinterpret_cast<const uint4*>(blob + p.v_off + (head + src) * row_bytes);
+  uint4* kd = reinterpret_cast<uint4*>(blob + (head + dst) * row_bytes);
+  uint4* vd = reinterpret_cast<uint4*>(blob + p.v_off + (head + dst) * row_bytes);
+  for (int i = lane; i < 2 * vec; i += 32) {
+    if (i < vec) kd[i] = ks[i];
+    else vd[i - vec] = vs[i - vec];
+  }
+  if (lane == 0) {
+    int* pp = reinterpret_cast<int*>(blob + p.pos_off) + head;
+    pp[dst] = pp[src];
+  }
+}
+
+}  // namespace kvc

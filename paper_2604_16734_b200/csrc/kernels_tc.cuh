@@ -1,0 +1,324 @@
+// Tensor-core kernels for bf16 (sm_100a): attention (a1, Eq. 1) and score (a2, Eq. 4).
+// Operands are staged in shared memory by TMA in the 128-byte-swizzled layouts tcgen05.mma reads,
+// accumulators live in TMEM, and only the two dense contractions (Q K^T and P V) use the tensor
+// cores; softmax, masking and the score reduction run on the CUDA cores in fp32.
+#pragma once
+#include <cuda.h>
+#include "geom.cuh"
+#include "ptx.cuh"
+
+namespace kvc {
+
+static constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 bf16 (one 128-byte swizzled row each)
+
+// Row packing shared by both kernels: for kv-head g the G query heads that share it are stacked
+// with the tokens, row r = (token - tok0) * G + (head - g*G), so keys and values are read once per
+// kv-head.  A tile holds TOK = 128 / G tokens (TOK * G <= 128 rows).
+
+struct TcSmemAttn {
+  uint64_t bar_q, bar_kv, bar_s, bar_p, bar_o;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// ------------------------------------------------------------------------------------------------
+// a1 attention, one 128-row tile per CTA.
+// Warps 0-3: softmax (thread = one row = one TMEM lane).  Warp 4: one elected lane issues the TMA
+// loads and the MMAs.  Per 128-key tile: S = Q K^T (tcgen05, fp32 in TMEM) -> online softmax in
+// registers -> P (bf16) written back to TMEM over S -> O += P V (A operand from TMEM, V read
+// MN-major from shared memory).
+// grid (ceil(n / TOK), Hkv, nl), block 160, dynamic smem 3 * (D/64) * 16 KB + 1 KB alignment slack.
+template <int D>
+__global__ void __launch_bounds__(160) attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                      const __grid_constant__ CUtensorMap tm_k,
+                                                      const __grid_constant__ CUtensorMap tm_v,
+                                                      __nv_bfloat16* __restrict__ out, char* __restrict__ ws, Geom p) {
+  constexpr int NSUB = D / 64;
+  constexpr uint32_t TMEM_COLS = 256;          // S/P at columns [0,128), O at [128, 128 + D)
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sK = sQ + NSUB * kSubTileBytes;
+  uint8_t* sV = sK + NSUB * kSubTileBytes;
+  __shared__ TcSmemAttn sh;
+
+  const int layer = blockIdx.z, g = blockIdx.y;
+  const int TOK = 128 / p.G, rows = TOK * p.G;
+  const int tok0 = blockIdx.x * TOK;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int last_tok = min(tok0 + TOK, p.n) - 1;
+  const int kv_end = p.n_c + last_tok + 1;
+  const int n_tiles = (kv_end + 127) / 128;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sh.bar_q, 1); mbar_init(&sh.bar_kv, 1); mbar_init(&sh.bar_s, 1);
+    mbar_init(&sh.bar_p, 128); mbar_init(&sh.bar_o, 1);
+    sh.abort_flag = 0;
+    mbar_fence_init();
+  }
+  // rows of the Q tile that TMA never writes (rows >= TOK*G) must still be finite
+  for (int i = threadIdx.x; i < NSUB * (128 - rows) * 8; i += blockDim.x) {
+    const int sub = i / ((128 - rows) * 8), rem = i % ((128 - rows) * 8);
+    reinterpret_cast<uint4*>(sQ + sub * kSubTileBytes + rows * 128)[rem] = make_uint4(0, 0, 0, 0);
+  }
+  fence_proxy_async_smem();
+  if (warp == 4) {
+    tmem_alloc(&sh.tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sh.tmem_base;
+  const uint32_t tmem_S = tmem, tmem_O = tmem + 128;
+  volatile int* abort_flag = &sh.abort_flag;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
+      mbar_expect_tx(&sh.bar_q, NSUB * rows * 128);
+      for (int sub = 0; sub < NSUB; ++sub)
+        tma_load_4d(sQ + sub * kSubTileBytes, &tm_q, &sh.bar_q, sub * 64, g * p.G, tok0, layer);
+      const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
+      const uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
+      const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
+      bool ok = true;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        if (j > 0) ok = mbar_wait(&sh.bar_o, (j - 1) & 1, abort_flag);     // K/V smem and S/P TMEM free again
+        if (!ok) break;
+        mbar_expect_tx(&sh.bar_kv, 2 * NSUB * kSubTileBytes);
+        for (int sub = 0; sub < NSUB; ++sub) {
+          tma_load_4d(sK + sub * kSubTileBytes, &tm_k, &sh.bar_kv, sub * 64, j * 128, g, layer);
+          tma_load_4d(sV + sub * kSubTileBytes, &tm_v, &sh.bar_kv, sub * 64, j * 128, g, layer);
+        }
+        if (j == 0) ok = mbar_wait(&sh.bar_q, 0, abort_flag);
+        ok = ok && mbar_wait(&sh.bar_kv, j & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {                 // S = Q K^T, 16 of the d columns per MMA
+          const uint32_t off = (kk / 4) * kSubTileBytes + (kk % 4) * 32;
+          mma_ss(tmem_S, smem_desc_sw128(aQ + off, 16, 1024), smem_desc_sw128(aK + off, 16, 1024), idesc_qk,
+                 kk > 0);
+        }
+        mma_commit(&sh.bar_s);
+        ok = mbar_wait(&sh.bar_p, j & 1, abort_flag);         // P is in TMEM
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)                        // O += P V, 16 keys per MMA
+          mma_ts(tmem_O, tmem_S + kk * 8, smem_desc_sw128(aV + kk * 2048, kSubTileBytes, 1024), idesc_pv,
+                 (j > 0 || kk > 0));
+        mma_commit(&sh.bar_o);
+      }
+    }
+    __syncwarp();
+  } else {
+    const int r = threadIdx.x;                                // row of the tile = TMEM lane
+    const int tok = tok0 + r / p.G, hh = r % p.G;
+    const bool row_valid = r < rows && tok < p.n;
+    const int limit = p.n_c + tok + 1;                        // keys [0, limit) are visible to this row
+    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      ok = mbar_wait(&sh.bar_s, j & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after_sync();
+      uint32_t sr[128];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tmem_S + lane_addr + c * 32, sr + c * 32);
+      tmem_wait_ld();
+      const int lim = limit - j * 128;                        // columns [0, lim) of this tile are visible
+      float tmax = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 128; ++c) {
+        float t = __uint_as_float(sr[c]) * p.scale_log2;
+        t = c < lim ? t : -INFINITY;
+        sr[c] = __float_as_uint(t);
+        tmax = fmaxf(tmax, t);
+      }
+      const float m_new = fmaxf(m, tmax);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;   // fully masked so far: every p is 0
+      const float corr = fast_exp2(m - m_use);
+      float psum = 0.f;
+      uint32_t pk[64];
+#pragma unroll
+      for (int c = 0; c < 64; ++c) {
+        const float p0 = fast_exp2(__uint_as_float(sr[2 * c]) - m_use);
+        const float p1 = fast_exp2(__uint_as_float(sr[2 * c + 1]) - m_use);
+        psum += p0 + p1;
+        pk[c] = pack_bf16x2(p0, p1);
+      }
+      l = l * corr + psum;
+      m = m_new;
+      if (j > 0) {                                            // rescale the running output
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tmem_O + lane_addr + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+          tmem_st32(tmem_O + lane_addr + c * 32, o);
+        }
+      }
+      tmem_st32(tmem_S + lane_addr, pk);
+      tmem_st32(tmem_S + lane_addr + 32, pk + 32);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(&sh.bar_p);
+    }
+    if (ok) ok = mbar_wait(&sh.bar_o, (n_tiles - 1) & 1, abort_flag);
+    if (ok) {
+      tc_fence_after_sync();
+      const float inv = 1.f / l;
+      __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tmem_O + lane_addr + c * 32, o);
+        tmem_wait_ld();
+        if (row_valid) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 vv;
+            vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+            vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+            vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+            vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+            reinterpret_cast<uint4*>(orow + c * 32)[i] = vv;
+          }
+        }
+      }
+      if (row_valid) {
+        float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
+        lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m + log2f(l)) * 0.6931471805599453f;
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+}
+
+// ------------------------------------------------------------------------------------------------
+// a2 score: one CTA per 128 candidate keys of one kv-head.  S^T = K_tile Q_obs^T puts keys on the
+// TMEM lanes, so each thread owns one key and sums 2^(s*scale_log2 - lse2) over the observer
+// columns in its own registers.  Observer rows are processed in groups of up to 256 columns.
+// grid (ceil(n_cand/128), Hkv, nl), block 128, dynamic smem (D/64)*16 KB + (D/64)*32 KB + 1 KB.
+struct TcSmemScore {
+  uint64_t bar_k, bar_q, bar_s;
+  uint32_t tmem_base;
+  int abort_flag;
+  float lse2[256];
+};
+
+template <int D>
+__global__ void __launch_bounds__(128) score_tc_kernel(const __grid_constant__ CUtensorMap tm_k,
+                                                       const __grid_constant__ CUtensorMap tm_qobs,
+                                                       char* __restrict__ ws, Geom p, int tok_per_group) {
+  constexpr int NSUB = D / 64;
+  constexpr uint32_t TMEM_COLS = 256;
+  constexpr int kQSubBytes = 256 * 128;        // up to 256 observer rows x 128 B
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sK = smem;
+  uint8_t* sQ = sK + NSUB * kSubTileBytes;
+  __shared__ TcSmemScore sh;
+
+  const int layer = blockIdx.z, g = blockIdx.y, key0 = blockIdx.x * 128;
+  const int warp = threadIdx.x >> 5;
+  char* slot = ws_slot(ws, p, layer);
+  const float* lse = reinterpret_cast<const float*>(slot + p.lse_off);
+  float* score = reinterpret_cast<float*>(slot + p.score_off) + static_cast<long long>(g) * p.cap;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sh.bar_k, 1); mbar_init(&sh.bar_q, 1); mbar_init(&sh.bar_s, 1);
+    sh.abort_flag = 0;
+    mbar_fence_init();
+  }
+  // observer rows beyond the last group's real rows are padding: keep them finite
+  for (int i = threadIdx.x; i < NSUB * kQSubBytes / 16; i += blockDim.x)
+    reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
+  fence_proxy_async_smem();
+  if (warp == 0) {
+    tmem_alloc(&sh.tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sh.tmem_base;
+  volatile int* abort_flag = &sh.abort_flag;
+  const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_qobs);
+    mbar_expect_tx(&sh.bar_k, NSUB * kSubTileBytes);
+    for (int sub = 0; sub < NSUB; ++sub)
+      tma_load_4d(sK + sub * kSubTileBytes, &tm_k, &sh.bar_k, sub * 64, key0, g, layer);
+  }
+  float acc = 0.f;
+  bool ok = true;
+  const int n_groups = (p.w + tok_per_group - 1) / tok_per_group;
+  for (int grp = 0; grp < n_groups && ok; ++grp) {
+    const int t_first = p.n - p.w + grp * tok_per_group;               // first observer token of the group
+    const int t_cnt = min(tok_per_group, p.n - t_first);
+    const int cols = t_cnt * p.G;                                      // real observer columns
+    const int n_mma = (cols + 15) & ~15;                               // MMA N: multiple of 16, <= 256
+    // everyone is past the previous group's TMEM reads and smem reads
+    tc_fence_before_sync();
+    __syncthreads();
+    for (int c = threadIdx.x; c < 256; c += blockDim.x) {
+      float lv = INFINITY;                                             // padding column: 2^-inf = 0
+      if (c < cols) lv = lse[static_cast<long long>(t_first + c / p.G) * p.Hq + g * p.G + c % p.G] * 1.4426950408889634f;
+      sh.lse2[c] = lv;
+    }
+    if (threadIdx.x == 0) {
+      // the box always spans tok_per_group tokens; tokens past n are zero-filled by TMA
+      mbar_expect_tx(&sh.bar_q, NSUB * tok_per_group * p.G * 128);
+      for (int sub = 0; sub < NSUB; ++sub)
+        tma_load_4d(sQ + sub * kQSubBytes, &tm_qobs, &sh.bar_q, sub * 64, g * p.G, t_first, layer);
+      if (grp == 0) ok = mbar_wait(&sh.bar_k, 0, abort_flag);
+      ok = ok && mbar_wait(&sh.bar_q, grp & 1, abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        const uint32_t idesc = idesc_bf16_f32(128, n_mma, 0, 0);
+        const uint32_t aK = smem_u32(sK), aQ = smem_u32(sQ);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+          mma_ss(tmem, smem_desc_sw128(aK + (kk / 4) * kSubTileBytes + (kk % 4) * 32, 16, 1024),
+                 smem_desc_sw128(aQ + (kk / 4) * kQSubBytes + (kk % 4) * 32, 16, 1024), idesc, kk > 0);
+        mma_commit(&sh.bar_s);
+      }
+    }
+    __syncwarp();
+    __syncthreads();                                                   // lse2 visible
+    ok = mbar_wait(&sh.bar_s, grp & 1, abort_flag);
+    if (!ok) break;
+    tc_fence_after_sync();
+    for (int c0 = 0; c0 < n_mma; c0 += 16) {
+      uint32_t sr[16];
+      tmem_ld16(tmem + lane_addr + c0, sr);
+      tmem_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) acc += fast_exp2(__uint_as_float(sr[i]) * p.scale_log2 - sh.lse2[c0 + i]);
+    }
+  }
+  const int key = key0 + threadIdx.x;
+  if (ok && key < p.n_cand) score[key] = acc;
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+}
+
+}  // namespace kvc

@@ -1,0 +1,436 @@
+// Host side of the kvc C ABI (see include/kvc.h): argument checks, launch geometry, TMA tensor
+// maps, kernel launches on the caller's stream.  Allocates no device memory.
+#include "../../include/kvc.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdarg.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "geom.cuh"
+#include "kernels_cc.cuh"
+#include "kernels_tc.cuh"
+
+using kvc::Geom;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct kvc_ctx {
+  uint32_t magic;
+  kvc_config cfg;
+  int G, cap, w_cfg;
+  float scale;
+  size_t elem, blob_bytes, v_off, pos_off;
+  size_t ws_slot_bytes, ws_bytes, lse_off, score_off, msrc_off, mdst_off, mcount_off;
+  std::vector<int> len;          // current cache length per layer, -1 = never reset
+  long long launches;
+  EncodeTiledFn encode;
+  bool use_tc;
+  char err[512];
+};
+
+static const uint32_t kMagic = 0x6b766331u;   // "kvc1"
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static int fail(kvc_ctx* c, int code, const char* fmt, ...) {
+  if (c) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c->err, sizeof(c->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+static bool live(const kvc_ctx* c) { return c && c->magic == kMagic; }
+
+extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
+  if (!out) return KVC_EINVAL;
+  *out = nullptr;
+  if (!cfg) return KVC_EINVAL;
+  if (cfg->n_layers < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads < 1) return KVC_EINVAL;
+  if (cfg->n_q_heads % cfg->n_kv_heads != 0) return KVC_EINVAL;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVC_EINVAL;
+  if (cfg->dtype != KVC_F32 && cfg->dtype != KVC_BF16) return KVC_EINVAL;
+  if (cfg->budget < 1 || cfg->max_chunk < 1) return KVC_EINVAL;
+  if (cfg->policy != KVC_SCORE_ATTN) return KVC_EINVAL;
+  if (cfg->obs_window < 0) return KVC_EINVAL;
+  if (!(cfg->softmax_scale >= 0.f) || isinf(cfg->softmax_scale)) return KVC_EINVAL;
+  const int w = cfg->obs_window == 0 ? 32 : cfg->obs_window;
+  if (w > cfg->budget) return KVC_EINVAL;                 // the protected window must fit the budget
+  const int G = cfg->n_q_heads / cfg->n_kv_heads;
+  if (G > 128) return KVC_EINVAL;
+  if (cfg->device < 0) return KVC_EINVAL;
+  if ((long long)cfg->budget + cfg->max_chunk > (1ll << 30)) return KVC_EINVAL;
+
+  kvc_ctx* c = new (std::nothrow) kvc_ctx();
+  if (!c) return KVC_EINVAL;
+  c->magic = kMagic;
+  c->cfg = *cfg;
+  c->G = G;
+  c->w_cfg = w;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+  c->cap = (int)align_up((size_t)cfg->budget + cfg->max_chunk, 128);
+  c->elem = cfg->dtype == KVC_F32 ? 4 : 2;
+  const size_t kv_bytes = (size_t)cfg->n_kv_heads * c->cap * cfg->head_dim * c->elem;
+  c->v_off = kv_bytes;
+  c->pos_off = 2 * kv_bytes;
+  c->blob_bytes = align_up(2 * kv_bytes + (size_t)cfg->n_kv_heads * c->cap * 4, 1024);
+  size_t o = 0;
+  c->lse_off = o;    o = align_up(o + (size_t)cfg->max_chunk * cfg->n_q_heads * 4, 256);
+  c->score_off = o;  o = align_up(o + (size_t)cfg->n_kv_heads * c->cap * 4, 256);
+  c->msrc_off = o;   o = align_up(o + (size_t)cfg->n_kv_heads * cfg->max_chunk * 4, 256);
+  c->mdst_off = o;   o = align_up(o + (size_t)cfg->n_kv_heads * cfg->max_chunk * 4, 256);
+  c->mcount_off = o; o = align_up(o + (size_t)cfg->n_kv_heads * 4, 256);
+  c->ws_slot_bytes = o;
+  c->ws_bytes = kvc::kWsHeaderBytes + o * cfg->n_layers;
+  c->len.assign(cfg->n_layers, -1);
+  c->launches = 0;
+  c->encode = nullptr;
+  c->use_tc = cfg->dtype == KVC_BF16 && !(cfg->flags & KVC_FLAG_CUDA_CORES);
+  c->err[0] = 0;
+  *out = c;
+  return KVC_OK;
+}
+
+extern "C" int kvc_destroy(kvc_ctx* c) {
+  if (!live(c)) return KVC_ESTATE;
+  c->magic = 0;
+  delete c;
+  return KVC_OK;
+}
+
+extern "C" const char* kvc_last_error(const kvc_ctx* c) { return live(c) ? c->err : "invalid context"; }
+extern "C" long long kvc_launch_count(const kvc_ctx* c) { return live(c) ? c->launches : -1; }
+
+extern "C" int kvc_cache_nbytes(const kvc_ctx* c, size_t* per_layer, size_t* workspace) {
+  if (!live(c)) return KVC_ESTATE;
+  if (per_layer) *per_layer = c->blob_bytes;
+  if (workspace) *workspace = c->ws_bytes;
+  return KVC_OK;
+}
+
+extern "C" int kvc_kv_bytes(const kvc_ctx* c, long long seq_len, size_t* logical, size_t* physical,
+                            size_t* uncompressed) {
+  if (!live(c)) return KVC_ESTATE;
+  if (seq_len < 0) return KVC_EINVAL;
+  // Eq. 2: 2 x layers x heads x dim_head x precision x sequence length
+  const size_t per_tok = 2 * (size_t)c->cfg.n_layers * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
+  if (logical) *logical = per_tok * c->cfg.budget;
+  if (physical) *physical = per_tok * c->cap;
+  if (uncompressed) *uncompressed = per_tok * (size_t)seq_len;
+  return KVC_OK;
+}
+
+static int check_cuda(kvc_ctx* c, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return KVC_OK;
+  return fail(c, KVC_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+extern "C" int kvc_reset(kvc_ctx* c, int layer, int n_layers, void* cache, size_t cache_layer_stride, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (layer < 0 || n_layers < 1 || layer + n_layers > c->cfg.n_layers) return fail(c, KVC_EINVAL, "layer range");
+  if (!cache || !aligned16(cache)) return fail(c, KVC_EINVAL, "cache pointer null or misaligned");
+  if (n_layers > 1 && (cache_layer_stride < c->blob_bytes || cache_layer_stride % 16)) return fail(c, KVC_EINVAL, "cache_layer_stride");
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int i = 0; i < n_layers; ++i) {
+    int rc = check_cuda(c, cudaMemsetAsync((char*)cache + (size_t)i * cache_layer_stride, 0, c->blob_bytes, st), "cudaMemsetAsync");
+    if (rc) return rc;
+    c->len[layer + i] = 0;
+  }
+  return KVC_OK;
+}
+
+extern "C" int kvc_workspace_init(kvc_ctx* c, void* workspace, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!workspace || !aligned16(workspace)) return fail(c, KVC_EINVAL, "workspace pointer null or misaligned");
+  return check_cuda(c, cudaMemsetAsync(workspace, 0, kvc::kWsHeaderBytes, (cudaStream_t)stream), "cudaMemsetAsync");
+}
+
+extern "C" int kvc_cache_view(const kvc_ctx* c, int layer, void* cache, kvc_view* v) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!v || !cache || layer < 0 || layer >= c->cfg.n_layers) return KVC_EINVAL;
+  if (c->len[layer] < 0) return KVC_ESTATE;
+  v->k = cache;
+  v->v = (char*)cache + c->v_off;
+  v->pos = (int*)((char*)cache + c->pos_off);
+  v->len = c->len[layer];
+  v->cap = c->cap;
+  v->n_kv_heads = c->cfg.n_kv_heads;
+  v->head_dim = c->cfg.head_dim;
+  v->dtype = c->cfg.dtype;
+  return KVC_OK;
+}
+
+extern "C" int kvc_workspace_view(const kvc_ctx* c, void* workspace, int slot, float** lse, float** score) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!workspace || slot < 0 || slot >= c->cfg.n_layers) return KVC_EINVAL;
+  char* s = (char*)workspace + kvc::kWsHeaderBytes + (size_t)slot * c->ws_slot_bytes;
+  if (lse) *lse = (float*)(s + c->lse_off);
+  if (score) *score = (float*)(s + c->score_off);
+  return KVC_OK;
+}
+
+extern "C" int kvc_status(kvc_ctx* c, void* workspace, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!workspace) return KVC_EINVAL;
+  int word = 0;
+  int rc = check_cuda(c, cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream), "cudaMemcpyAsync");
+  if (rc) return rc;
+  rc = check_cuda(c, cudaStreamSynchronize((cudaStream_t)stream), "cudaStreamSynchronize");
+  if (rc) return rc;
+  if (word != 0) return fail(c, word == KVC_ETIMEOUT ? KVC_ETIMEOUT : KVC_ECUDA, "device status word %d", word);
+  return KVC_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+static int get_encoder(kvc_ctx* c) {
+  if (c->encode) return KVC_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+    return fail(c, KVC_ECUDA, "cuTensorMapEncodeTiled entry point unavailable: %s", cudaGetErrorString(e));
+  c->encode = (EncodeTiledFn)fn;
+  return KVC_OK;
+}
+
+// bf16 4-D tensor map with 128-byte swizzle; dims/box innermost first, strides in bytes for dims 1..3.
+static int make_map(kvc_ctx* c, CUtensorMap* m, const void* base, const uint64_t dims[4], const uint64_t strides[3],
+                    const uint32_t box[4]) {
+  cuuint64_t gd[4] = {dims[0], dims[1], dims[2], dims[3]};
+  cuuint64_t gs[3] = {strides[0], strides[1], strides[2]};
+  cuuint32_t bx[4] = {box[0], box[1], box[2], box[3]};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gd, gs, bx, es,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(c, KVC_ECUDA, "cuTensorMapEncodeTiled failed (%d): dims %llu %llu %llu %llu box %u %u %u %u", (int)r,
+                (unsigned long long)dims[0], (unsigned long long)dims[1], (unsigned long long)dims[2],
+                (unsigned long long)dims[3], box[0], box[1], box[2], box[3]);
+  return KVC_OK;
+}
+
+template <typename T, int D>
+static void launch_cc_attn(const Geom& g, const void* q, void* cache, void* out, void* ws, cudaStream_t st) {
+  dim3 grid((g.n + 15) / 16, g.Hq, g.nl);
+  kvc::attn_cc_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const char*)cache, (T*)out, (char*)ws, g);
+}
+template <typename T, int D>
+static cudaError_t launch_cc_score(const Geom& g, const void* q, void* cache, void* ws, cudaStream_t st) {
+  const int smem = (128 * (D + 4) + 32 * D + 32) * 4;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kvc::score_cc_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  dim3 grid((g.n_cand + 127) / 128, g.Hkv, g.nl);
+  kvc::score_cc_kernel<T, D><<<grid, 128, smem, st>>>((const T*)q, (const char*)cache, (char*)ws, g);
+  return cudaSuccess;
+}
+
+template <int D>
+static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                  void* out, void* ws, cudaStream_t st) {
+  const int smem = 3 * (D / 64) * kvc::kSubTileBytes + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int TOK = 128 / g.G;
+  dim3 grid((g.n + TOK - 1) / TOK, g.Hkv, g.nl);
+  kvc::attn_tc_kernel<D><<<grid, 160, smem, st>>>(tq, tk, tv, (__nv_bfloat16*)out, (char*)ws, g);
+  return cudaSuccess;
+}
+template <int D>
+static cudaError_t launch_tc_score(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* ws,
+                                   int tok_per_group, cudaStream_t st) {
+  const int smem = (D / 64) * (kvc::kSubTileBytes + 256 * 128) + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kvc::score_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  dim3 grid((g.n_cand + 127) / 128, g.Hkv, g.nl);
+  kvc::score_tc_kernel<D><<<grid, 128, smem, st>>>(tk, tqo, (char*)ws, g, tok_per_group);
+  return cudaSuccess;
+}
+
+static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_ls, const void* k, const void* v,
+                     long long kv_ls, int n, long long pos0, void* cache, size_t cache_ls, void* ws, void* out,
+                     long long out_ls, cudaStream_t st) {
+  const kvc_config& cf = c->cfg;
+  if (layer0 < 0 || nl < 1 || layer0 + nl > cf.n_layers) return fail(c, KVC_EINVAL, "layer range [%d, %d) outside [0, %d)", layer0, layer0 + nl, cf.n_layers);
+  if (!q || !k || !v || !cache || !ws || !out) return fail(c, KVC_EINVAL, "null pointer argument");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(cache) || !aligned16(ws) || !aligned16(out))
+    return fail(c, KVC_EINVAL, "pointers must be 16-byte aligned");
+  if (n < 1 || n > cf.max_chunk) return fail(c, KVC_EINVAL, "n = %d outside [1, max_chunk = %d]", n, cf.max_chunk);
+  if (pos0 < 0 || pos0 + n > 0x7fffffffLL) return fail(c, KVC_EINVAL, "pos0 out of range");
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != cf.device)
+    return fail(c, KVC_ESTATE, "current CUDA device %d is not the context's device %d", dev, cf.device);
+  const int n_c = c->len[layer0];
+  for (int i = 0; i < nl; ++i) {
+    if (c->len[layer0 + i] < 0) return fail(c, KVC_ESTATE, "layer %d used before kvc_reset", layer0 + i);
+    if (c->len[layer0 + i] != n_c) return fail(c, KVC_ESTATE, "batched layers hold different cache lengths");
+  }
+  if (nl > 1) {
+    const long long qmin = (long long)n * cf.n_q_heads * cf.head_dim, kmin = (long long)n * cf.n_kv_heads * cf.head_dim;
+    if (q_ls < qmin || out_ls < qmin || kv_ls < kmin || cache_ls < c->blob_bytes)
+      return fail(c, KVC_EINVAL, "layer strides too small");
+    if ((q_ls * c->elem) % 16 || (out_ls * c->elem) % 16 || (kv_ls * c->elem) % 16 || cache_ls % 16)
+      return fail(c, KVC_EINVAL, "layer strides must be multiples of 16 bytes");
+  } else {
+    q_ls = out_ls = (long long)n * cf.n_q_heads * cf.head_dim;
+    kv_ls = (long long)n * cf.n_kv_heads * cf.head_dim;
+    cache_ls = c->blob_bytes;
+  }
+
+  Geom g;
+  memset(&g, 0, sizeof(g));
+  g.n = n; g.n_c = n_c; g.tot = n_c + n; g.B = cf.budget;
+  g.w = c->w_cfg < n ? c->w_cfg : n;
+  g.G = c->G; g.Hq = cf.n_q_heads; g.Hkv = cf.n_kv_heads; g.d = cf.head_dim; g.cap = c->cap; g.nl = nl;
+  g.max_chunk = cf.max_chunk;
+  g.n_cand = g.tot - g.w; g.n_keep = g.B - g.w;
+  g.scale_log2 = c->scale * 1.4426950408889634f;
+  g.pos0 = pos0;
+  g.q_ls = q_ls; g.kv_ls = kv_ls; g.out_ls = out_ls; g.cache_ls = (long long)cache_ls;
+  g.v_off = (long long)c->v_off; g.pos_off = (long long)c->pos_off;
+  g.ws_ls = (long long)c->ws_slot_bytes;
+  g.lse_off = c->lse_off; g.score_off = c->score_off; g.msrc_off = c->msrc_off; g.mdst_off = c->mdst_off;
+  g.mcount_off = c->mcount_off;
+  const bool evict = g.tot > g.B;                      // Alg. 1: "if |C| > M"
+  const bool f32 = cf.dtype == KVC_F32;
+  const int D = cf.head_dim;
+
+  // tensor maps first: nothing is enqueued if an encode fails
+  CUtensorMap tq, tk, tv, tqo;
+  int tok_per_group = 0;
+  if (c->use_tc) {
+    int rc = get_encoder(c);
+    if (rc) return rc;
+    const int TOK = 128 / g.G;
+    const uint64_t qd[4] = {(uint64_t)D, (uint64_t)g.Hq, (uint64_t)n, (uint64_t)nl};
+    const uint64_t qs[3] = {(uint64_t)D * 2, (uint64_t)g.Hq * D * 2, (uint64_t)q_ls * 2};
+    const uint32_t qb[4] = {64, (uint32_t)g.G, (uint32_t)TOK, 1};
+    if ((rc = make_map(c, &tq, q, qd, qs, qb))) return rc;
+    const uint64_t kd[4] = {(uint64_t)D, (uint64_t)g.cap, (uint64_t)g.Hkv, (uint64_t)nl};
+    const uint64_t ks[3] = {(uint64_t)D * 2, (uint64_t)g.cap * D * 2, (uint64_t)cache_ls};
+    const uint32_t kb[4] = {64, 128, 1, 1};
+    if ((rc = make_map(c, &tk, cache, kd, ks, kb))) return rc;
+    if ((rc = make_map(c, &tv, (char*)cache + c->v_off, kd, ks, kb))) return rc;
+    if (evict) {
+      tok_per_group = 256 / g.G;
+      if (tok_per_group > g.w) tok_per_group = g.w;
+      const uint32_t ob[4] = {64, (uint32_t)g.G, (uint32_t)tok_per_group, 1};
+      if ((rc = make_map(c, &tqo, q, qd, qs, ob))) return rc;
+    }
+  }
+
+  // a0 append
+  {
+    dim3 grid((n * g.Hkv + 7) / 8, 1, nl);
+    if (f32) kvc::append_kernel<float><<<grid, 256, 0, st>>>((const float*)k, (const float*)v, (char*)cache, g);
+    else kvc::append_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (char*)cache, g);
+    c->launches++;
+  }
+  // a1 attention
+  cudaError_t e = cudaSuccess;
+  if (c->use_tc) {
+    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, out, ws, st) : launch_tc_attn<64>(g, tq, tk, tv, out, ws, st);
+  } else if (f32) {
+    if (D == 128) launch_cc_attn<float, 128>(g, q, cache, out, ws, st); else launch_cc_attn<float, 64>(g, q, cache, out, ws, st);
+  } else {
+    if (D == 128) launch_cc_attn<__nv_bfloat16, 128>(g, q, cache, out, ws, st); else launch_cc_attn<__nv_bfloat16, 64>(g, q, cache, out, ws, st);
+  }
+  if (e != cudaSuccess) return check_cuda(c, e, "attention launch setup");
+  c->launches++;
+  if (evict) {
+    // a2 score
+    if (c->use_tc) {
+      e = D == 128 ? launch_tc_score<128>(g, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, tk, tqo, ws, tok_per_group, st);
+    } else if (f32) {
+      e = D == 128 ? launch_cc_score<float, 128>(g, q, cache, ws, st) : launch_cc_score<float, 64>(g, q, cache, ws, st);
+    } else {
+      e = D == 128 ? launch_cc_score<__nv_bfloat16, 128>(g, q, cache, ws, st) : launch_cc_score<__nv_bfloat16, 64>(g, q, cache, ws, st);
+    }
+    if (e != cudaSuccess) return check_cuda(c, e, "score launch setup");
+    c->launches++;
+    // a3 select
+    kvc::select_kernel<<<dim3(g.Hkv, 1, nl), 1024, 0, st>>>((const char*)cache, (char*)ws, g);
+    c->launches++;
+    // a4 compact: at most min(n, tot - B) entries sit at or above row B
+    const int max_moves = n < g.tot - g.B ? n : g.tot - g.B;
+    kvc::compact_kernel<<<dim3((max_moves + 7) / 8, g.Hkv, nl), 256, 0, st>>>((char*)cache, (const char*)ws, g, (int)c->elem);
+    c->launches++;
+  }
+  int rc = check_cuda(c, cudaGetLastError(), "kernel launch");
+  if (rc) return rc;
+  const int new_len = evict ? g.B : g.tot;
+  for (int i = 0; i < nl; ++i) c->len[layer0 + i] = new_len;
+  return KVC_OK;
+}
+
+extern "C" int kvc_prefill_chunk(kvc_ctx* c, int layer, const void* q, const void* k, const void* v, int n,
+                                 long long pos0, void* cache, void* workspace, void* out, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, workspace, out, 0, (cudaStream_t)stream);
+}
+
+extern "C" int kvc_prefill_chunk_layers(kvc_ctx* c, int layer0, int n_layers, const void* q, long long q_layer_stride,
+                                        const void* k, const void* v, long long kv_layer_stride, int n, long long pos0,
+                                        void* cache, size_t cache_layer_stride, void* workspace, void* out,
+                                        long long out_layer_stride, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  return run_chunk(c, layer0, n_layers, q, q_layer_stride, k, v, kv_layer_stride, n, pos0, cache, cache_layer_stride,
+                   workspace, out, out_layer_stride, (cudaStream_t)stream);
+}
+
+extern "C" int kvc_staging_nbytes(const kvc_ctx* c, size_t* nbytes) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!nbytes) return KVC_EINVAL;
+  const size_t qb = (size_t)c->cfg.max_chunk * c->cfg.n_q_heads * c->cfg.head_dim * c->elem;
+  const size_t kb = (size_t)c->cfg.max_chunk * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
+  *nbytes = 2 * align_up(qb, 256) + 2 * align_up(kb, 256);
+  return KVC_OK;
+}
+
+extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host, const void* k_host, const void* v_host,
+                                      int n, long long pos0, void* cache, void* workspace, void* staging, void* out_host,
+                                      void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!q_host || !k_host || !v_host || !out_host || !staging) return fail(c, KVC_EINVAL, "null pointer argument");
+  if (n < 1 || n > c->cfg.max_chunk) return fail(c, KVC_EINVAL, "n = %d outside [1, max_chunk = %d]", n, c->cfg.max_chunk);
+  if (!aligned16(staging)) return fail(c, KVC_EINVAL, "staging must be 16-byte aligned");
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t qb = (size_t)n * c->cfg.n_q_heads * c->cfg.head_dim * c->elem;
+  const size_t kb = (size_t)n * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
+  char* dq = (char*)staging;
+  char* dk = dq + align_up(qb, 256);
+  char* dv = dk + align_up(kb, 256);
+  char* dout = dv + align_up(kb, 256);
+  int rc;
+  if ((rc = check_cuda(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st), "H2D q"))) return rc;
+  if ((rc = check_cuda(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, st), "H2D k"))) return rc;
+  if ((rc = check_cuda(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, st), "H2D v"))) return rc;
+  rc = run_chunk(c, layer, 1, dq, 0, dk, dv, 0, n, pos0, cache, 0, workspace, dout, 0, st);
+  if (rc) return rc;
+  return check_cuda(c, cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st), "D2H out");
+}

@@ -1,0 +1,213 @@
+"""Parity of the CUDA library (through the C ABI) against the fp64 CPU oracle on the same seeded
+inputs.  Index sets must match bit-exactly unless the oracle's cut-off gap is below 1e-3; retained
+K/V rows must be bit-exact copies; attention outputs within 1e-4 (fp32) / 2e-2 (bf16) max-abs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_16734_b200 import binding
+from paper_2604_16734_b200.binding import Kvc, KvcError, KVC_FLAG_CUDA_CORES, KVC_EINVAL, KVC_ESTATE
+from paper_2604_16734_b200.workloads import CONFIGS, Workload, reduced
+
+from parity_util import compare_chunk, make_oracle, run_workload_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _kvc_for(cfg, flags=0, n_layers=None, max_chunk=None, budget=None):
+    return Kvc(cfg.n_layers if n_layers is None else n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
+               cfg.torch_dtype, cfg.budget if budget is None else budget,
+               cfg.chunk if max_chunk is None else max_chunk, cfg.obs_window, flags=flags)
+
+
+def _layers(cfg, layers):
+    wl = Workload(cfg)
+    return {l: wl.layer(l) for l in layers}
+
+
+# ------------------------------------------------------------------------------------------------
+# the benchmark's configurations (reduced in layers / frames so the oracle finishes in seconds)
+
+def test_c1_fp32_full():
+    cfg = CONFIGS["C1"]
+    kvc = _kvc_for(cfg)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0])
+    assert worst["err_out"] <= 1e-4
+    kvc.reset()
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], teacher_forced=True)
+    assert worst["err_out"] <= 1e-4 and worst["adopted"] == 0
+
+
+@pytest.mark.parametrize("flags", [0, KVC_FLAG_CUDA_CORES])
+def test_c2_llava_shaped_two_layers(flags):
+    cfg = reduced(CONFIGS["C2"], n_layers=2)
+    kvc = _kvc_for(cfg, flags)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0, 1]), [0, 1])
+    assert worst["err_out"] <= 2e-2
+
+
+@pytest.mark.parametrize("flags", [0, KVC_FLAG_CUDA_CORES])
+def test_c3_tiled_group_of_seven(flags):
+    cfg = reduced(CONFIGS["C3"], n_layers=1, n_units=2)       # 2 tiles of 576 + 128 text, B = 1024, G = 7
+    kvc = _kvc_for(cfg, flags)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0])
+    assert worst["err_out"] <= 2e-2
+
+
+def test_c4_video_frames():
+    cfg = reduced(CONFIGS["C4"], n_layers=1, n_units=12)      # 12 frames of 196 -> 2352 > B = 2048
+    kvc = _kvc_for(cfg)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0])
+    assert worst["err_out"] <= 2e-2
+    kvc.reset()
+    run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], teacher_forced=True)
+
+
+def test_c5_long_video_blocks():
+    cfg = reduced(CONFIGS["C5"], n_layers=1, n_units=36)      # 5184 vision tokens -> 6 blocks, B = 4096
+    kvc = _kvc_for(cfg)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=[0, 7])
+    assert worst["err_out"] <= 2e-2
+
+
+# ------------------------------------------------------------------------------------------------
+# ragged shapes and degenerate cases
+
+@pytest.mark.parametrize("dtype,d,hq,hkv,flags", [
+    (torch.float32, 64, 4, 1, 0), (torch.float32, 128, 6, 2, 0),
+    (torch.bfloat16, 128, 8, 2, 0), (torch.bfloat16, 64, 4, 4, 0), (torch.bfloat16, 128, 3, 1, 0),
+    (torch.bfloat16, 128, 8, 2, KVC_FLAG_CUDA_CORES),
+])
+def test_ragged_blocks(dtype, d, hq, hkv, flags):
+    torch.manual_seed(7)
+    B, c, w = 160, 200, 16
+    sizes = [1, 31, 128, 1, 200, 7, 129, 33, 160, 2, 16, 15]          # tot == B and tot == B + 1 both occur
+    kvc = Kvc(1, hq, hkv, d, dtype, B, c, w, flags=flags)
+    from oracle.kvc_oracle import KVCOracle
+    orc = KVCOracle(1, hq, hkv, d, B, w)
+    p = 0
+    for n in sizes:
+        q = torch.randn(n, hq, d).to(dtype); k = torch.randn(n, hkv, d).to(dtype); v = torch.randn(n, hkv, d).to(dtype)
+        compare_chunk(kvc, orc, 0, q, k, v, p)
+        p += n
+
+
+def test_first_block_larger_than_budget_and_window_equal_to_budget():
+    torch.manual_seed(8)
+    hq, hkv, d = 4, 2, 128
+    from oracle.kvc_oracle import KVCOracle
+    # one block of 300 tokens into a budget of 64: "process first, compress later" special case
+    kvc = Kvc(1, hq, hkv, d, torch.bfloat16, 64, 300, 32)
+    orc = KVCOracle(1, hq, hkv, d, 64, 32)
+    for p, n in ((0, 300), (300, 300)):
+        q = torch.randn(n, hq, d).bfloat16(); k = torch.randn(n, hkv, d).bfloat16(); v = torch.randn(n, hkv, d).bfloat16()
+        compare_chunk(kvc, orc, 0, q, k, v, p)
+    # w == B: only the observers' own keys survive
+    kvc = Kvc(1, hq, hkv, d, torch.float32, 32, 64, 32)
+    orc = KVCOracle(1, hq, hkv, d, 32, 32)
+    for p, n in ((0, 64), (64, 40), (104, 64)):
+        q = torch.randn(n, hq, d); k = torch.randn(n, hkv, d); v = torch.randn(n, hkv, d)
+        compare_chunk(kvc, orc, 0, q, k, v, p)
+        _, _, pos, ln = kvc.cache_view(0)
+        assert ln == 32 and sorted(pos[0, :32].tolist()) == list(range(p + n - 32, p + n))
+
+
+def test_budget_not_smaller_than_sequence_is_dense_attention():
+    # Alg. 1 never evicts when M >= |S|: the chunked result equals dense causal attention (library SDPA)
+    torch.manual_seed(9)
+    n_tot, hq, hkv, d = 500, 4, 2, 128
+    q = torch.randn(n_tot, hq, d).bfloat16(); k = torch.randn(n_tot, hkv, d).bfloat16(); v = torch.randn(n_tot, hkv, d).bfloat16()
+    kvc = Kvc(1, hq, hkv, d, torch.bfloat16, 512, 128)
+    outs, p = [], 0
+    for n in (128, 100, 128, 17, 127):
+        outs.append(kvc.prefill_chunk(0, q[p:p + n].cuda(), k[p:p + n].cuda(), v[p:p + n].cuda(), p)); p += n
+    out = torch.cat(outs).float().cpu()
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        q.double().permute(1, 0, 2), k.double().permute(1, 0, 2).repeat_interleave(2, 0),
+        v.double().permute(1, 0, 2).repeat_interleave(2, 0), is_causal=True).permute(1, 0, 2)
+    assert (out.double() - ref).abs().max() <= 2e-2
+    assert kvc.cache_view(0)[3] == n_tot
+
+
+def test_duplicate_keys_tie_break_keeps_older():
+    torch.manual_seed(10)
+    hq = hkv = 1; d = 64
+    kvc = Kvc(1, hq, hkv, d, torch.float32, 8, 8, 1)
+    base = torch.randn(1, 1, d)
+    k = base.repeat(6, 1, 1).contiguous(); v = torch.randn(6, 1, d); q = torch.randn(6, 1, d)
+    kvc.prefill_chunk(0, q.cuda(), k.cuda(), v.cuda(), 0)
+    q2 = torch.randn(4, 1, d); k2 = torch.randn(4, 1, d) * 50; v2 = torch.randn(4, 1, d)
+    kvc.prefill_chunk(0, q2.cuda(), k2.cuda(), v2.cuda(), 6)
+    _, _, pos, ln = kvc.cache_view(0)
+    kept = sorted(p for p in pos[0, :ln].tolist() if p < 6)
+    assert ln == 8 and kept == list(range(len(kept)))       # identical scores: the older entries stay
+
+
+def test_layer_batched_call_matches_per_layer_calls():
+    cfg = reduced(CONFIGS["C4"], n_layers=3, n_units=11)
+    wl = Workload(cfg)
+    qs, ks, vs = zip(*[wl.layer(l) for l in range(3)])
+    Q = torch.stack(qs).cuda(); K = torch.stack(ks).cuda(); V = torch.stack(vs).cuda()
+    a = _kvc_for(cfg); b = _kvc_for(cfg)
+    out_a = torch.empty_like(Q); out_b = torch.empty_like(Q)
+    for pos0, n in cfg.chunks():
+        for l in range(3):
+            a.prefill_chunk(l, Q[l, pos0:pos0 + n], K[l, pos0:pos0 + n], V[l, pos0:pos0 + n], pos0,
+                            out_a[l, pos0:pos0 + n])
+        b.prefill_chunk_layers(0, Q[:, pos0:pos0 + n], K[:, pos0:pos0 + n], V[:, pos0:pos0 + n], pos0,
+                               out_b[:, pos0:pos0 + n])
+    torch.cuda.synchronize()
+    assert a.status() == 0 and b.status() == 0
+    assert torch.equal(out_a, out_b)
+    for l in range(3):
+        Ka, Va, Pa, la = a.cache_view(l); Kb, Vb, Pb, lb = b.cache_view(l)
+        assert la == lb == cfg.budget
+        assert torch.equal(Pa[:, :la], Pb[:, :lb]) and torch.equal(Ka[:, :la], Kb[:, :lb]) and torch.equal(Va[:, :la], Vb[:, :lb])
+
+
+def test_host_buffer_entry_point():
+    cfg = reduced(CONFIGS["C2"], n_layers=1)
+    q, k, v = Workload(cfg).layer(0)
+    a = _kvc_for(cfg); b = _kvc_for(cfg)
+    qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+    out_h = torch.empty_like(q).pin_memory()
+    for pos0, n in cfg.chunks():
+        ref = a.prefill_chunk(0, q[pos0:pos0 + n].cuda(), k[pos0:pos0 + n].cuda(), v[pos0:pos0 + n].cuda(), pos0)
+        b.prefill_chunk_host(0, qh[pos0:pos0 + n], kh[pos0:pos0 + n], vh[pos0:pos0 + n], pos0, out_h[pos0:pos0 + n])
+        torch.cuda.synchronize()
+        assert torch.equal(ref.cpu(), out_h[pos0:pos0 + n])
+    assert torch.equal(a.cache_view(0)[2], b.cache_view(0)[2])
+
+
+def test_argument_errors_enqueue_nothing():
+    kvc = Kvc(2, 4, 2, 128, torch.bfloat16, 64, 32)
+    q = torch.randn(33, 4, 128, device="cuda").bfloat16(); k = torch.randn(33, 2, 128, device="cuda").bfloat16()
+    before = kvc.launch_count()
+    with pytest.raises(KvcError) as e:
+        kvc.prefill_chunk(0, q, k, k, 0)                       # n > max_chunk
+    assert e.value.code == KVC_EINVAL
+    with pytest.raises(KvcError) as e:
+        kvc._check(kvc._lib.kvc_prefill_chunk(kvc._h, 5, q.data_ptr(), k.data_ptr(), k.data_ptr(), 8, 0,
+                                              kvc.cache[0].data_ptr(), kvc.workspace.data_ptr(), q.data_ptr(), 0))
+        # layer out of range
+    assert e.value.code == KVC_EINVAL
+    with pytest.raises(KvcError) as e:
+        kvc._check(kvc._lib.kvc_prefill_chunk(kvc._h, 0, q.data_ptr() + 2, k.data_ptr(), k.data_ptr(), 8, 0,
+                                              kvc.cache[0].data_ptr(), kvc.workspace.data_ptr(), q.data_ptr(), 0))
+    assert e.value.code == KVC_EINVAL                          # misaligned pointer
+    assert kvc.launch_count() == before
+    fresh = Kvc(1, 4, 2, 128, torch.bfloat16, 64, 32, allocate=False)
+    fresh.cache = torch.empty(1, fresh.blob_bytes, dtype=torch.uint8, device="cuda")
+    fresh.workspace = torch.zeros(fresh.ws_bytes, dtype=torch.uint8, device="cuda")
+    with pytest.raises(KvcError) as e:
+        fresh.prefill_chunk(0, q[:8], k[:8], k[:8], 0)         # never reset
+    assert e.value.code == KVC_ESTATE
+    assert kvc.status() == 0
+
+
+def test_kv_bytes_stay_at_the_budget_bound():
+    cfg = reduced(CONFIGS["C4"], n_layers=2, n_units=12)
+    kvc = _kvc_for(cfg)
+    logical, physical, full = kvc.kv_bytes(cfg.n_tokens)
+    assert physical <= kvc.blob_bytes * 2 and logical < physical < full
+    assert kvc.cache.numel() == 2 * kvc.blob_bytes          # nothing else is ever allocated for the cache

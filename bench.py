@@ -1,0 +1,469 @@
+#!/usr/bin/env python
+"""Benchmark of the block-wise prefill hot path (append, attention, score, select, compact).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--mode graph|direct|batched]
+  python bench.py --impl reference ...      # the CPU oracle as the reference arm
+
+One "step" is one pass of the whole hot path over one synthetic request: every block of the
+workload's prefix through every layer, starting from empty caches.  Prints ONE JSON line.
+
+Modes (all run the same kernels through the C ABI):
+  direct   one kvc_prefill_chunk call per (block, layer), issued from Python each step
+  graph    the same calls captured once into a CUDA graph and replayed (no host work per step)
+  batched  one kvc_prefill_chunk_layers call per block, the layer index in the launch grid
+           (possible only because the synthetic q/k/v of all layers exist up front)
+With N > 1 every rank runs an independent replica of the request on its own GPU: the path has no
+cross-GPU exchange, so there is no collective inside the timed region (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_16734_b200.workloads import CONFIGS, Workload  # noqa: E402
+
+METRIC = "prefill tokens/s (attn+compress) per layer"
+UNIT = "tokens/s/layer"
+STEPS = ("append", "attention", "score", "select", "compact")
+
+
+# ------------------------------------------------------------------------------------------------
+# peaks (roofline denominators)
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work of one launch (what the method itself has to move / compute)
+
+def work_of_call(cfg, n, n_c, moves_per_head=None):
+    """Bytes and FLOPs per step kind for ONE layer of one kvc_prefill_chunk call."""
+    Hq, Hkv, d, sz, B = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.elem_bytes, cfg.budget
+    tot = n_c + n
+    w = min(cfg.obs_window, n)
+    out = {}
+    out["append"] = dict(bytes=2 * 2 * n * d * sz * Hkv + 4 * n * Hkv, flops=0)
+    out["attention"] = dict(bytes=2 * tot * d * sz * Hkv + 2 * n * d * sz * Hq + 4 * Hq * n,
+                            flops=4 * Hq * d * (n * n_c + n * (n + 1) // 2))
+    if tot > B:
+        m = min(n, tot - B) * Hkv if moves_per_head is None else int(sum(moves_per_head))
+        out["score"] = dict(bytes=Hkv * (tot - w) * d * sz + Hq * w * d * sz + 4 * Hq * w + 4 * Hkv * (tot - w),
+                            flops=2 * Hq * w * d * (tot - w))
+        out["select"] = dict(bytes=2 * 4 * Hkv * (tot - w) + 8 * m, flops=0)
+        out["compact"] = dict(bytes=m * (2 * 2 * d * sz + 8 + 8), flops=0)
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        self.marks = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu=timestamp,{self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=self.file,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def mark(self):
+        self.marks.append(time.time())
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.file.flush()
+        rows = []
+        try:
+            with open(self.file.name) as f:
+                for line in f:
+                    parts = [x.strip() for x in line.split(",")]
+                    if len(parts) >= 10:
+                        rows.append(parts)
+        finally:
+            try:
+                os.unlink(self.file.name)
+            except OSError:
+                pass
+        return rows
+
+    def summary(self, rows, t0, t1):
+        import datetime
+        sel = []
+        for r in rows:
+            try:
+                ts = datetime.datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+            except ValueError:
+                continue
+            if t0 - 0.05 <= ts <= t1 + 0.05:
+                sel.append(r)
+        used = sel if sel else rows
+        if not used:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        sm = [float(r[2]) for r in used]
+        reasons = set()
+        for r in used:
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[6:10]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=float(used[0][3]), reasons=sorted(reasons),
+                    samples=len(sel), power_w_max=max(float(r[4]) for r in used))
+
+
+# ------------------------------------------------------------------------------------------------
+# the reference arm: the CPU oracle on a bounded sample
+
+def oracle_sample_plan(cfg):
+    """(layers, kv_heads, chunks) of the bounded sample the oracle runs per step."""
+    sched = cfg.chunks()
+    if cfg.name in ("C1", "C2"):
+        return [0], None, sched, "layer 0, all kv-heads, whole prefix"
+    if cfg.name == "C3":
+        return [0], [0], sched, "layer 0, kv-head 0 of 4, whole prefix (scaled by 4)"
+    # video: the per-block cost is flat once the cache is full; sample the first blocks past the budget
+    n_fill = next(i for i, (p, n) in enumerate(sched) if p + n > cfg.budget) + 3
+    return [0], [0], sched[:n_fill], f"layer 0, kv-head 0 of {cfg.n_kv_heads}, first {n_fill} blocks (scaled by {cfg.n_kv_heads})"
+
+
+def run_oracle_sample(cfg, tensors_cpu):
+    from oracle.kvc_oracle import KVCOracle
+    layers, heads, chunks, desc = oracle_sample_plan(cfg)
+    orc = KVCOracle(1, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.budget, cfg.obs_window)
+    q, k, v = tensors_cpu
+    t0 = time.perf_counter()
+    tokens = 0
+    for pos0, n in chunks:
+        orc.prefill_chunk(0, q[pos0:pos0 + n], k[pos0:pos0 + n], v[pos0:pos0 + n], pos0, kv_heads=heads)
+        tokens += n
+    dt = time.perf_counter() - t0
+    frac_heads = 1.0 if heads is None else len(heads) / cfg.n_kv_heads
+    return tokens * len(layers) * frac_heads / dt, dt, desc
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def reference_arm(args, cfg, rank):
+    if rank != 0:
+        return
+    import numpy as np
+    wl = Workload(cfg, device="cpu")
+    q, k, v = wl.layer(0)
+    tens = (q.double().numpy(), k.double().numpy(), v.double().numpy())
+    for _ in range(min(args.warmup, 1)):
+        run_oracle_sample(cfg, tens)
+    vals, times = [], []
+    desc = ""
+    for _ in range(args.steps):
+        val, dt, desc = run_oracle_sample(cfg, tens)
+        vals.append(val); times.append(dt)
+    value = sum(vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+
+class Runner:
+    def __init__(self, cfg, device_index, n_layers=None):
+        from paper_2604_16734_b200.binding import Kvc
+        self.cfg = cfg
+        self.L = cfg.n_layers if n_layers is None else n_layers
+        self.dev = torch.device("cuda", device_index)
+        wl = Workload(cfg, device=self.dev)
+        N = cfg.n_tokens
+        self.Q = torch.empty(self.L, N, cfg.n_q_heads, cfg.head_dim, dtype=cfg.torch_dtype, device=self.dev)
+        self.K = torch.empty(self.L, N, cfg.n_kv_heads, cfg.head_dim, dtype=cfg.torch_dtype, device=self.dev)
+        self.V = torch.empty_like(self.K)
+        for l in range(self.L):
+            q, k, v = wl.layer(l)
+            self.Q[l], self.K[l], self.V[l] = q, k, v
+        del wl
+        self.O = torch.empty_like(self.Q)
+        self.kvc = Kvc(self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk,
+                       cfg.obs_window, device=device_index)
+        self.sched = cfg.chunks()
+        # raw pointers of every (block, layer) slice, so the per-call host work is one ctypes call
+        self.ptrs = {}
+        for ci, (p, n) in enumerate(self.sched):
+            for l in range(self.L):
+                self.ptrs[ci, l] = (self.Q[l, p:p + n].data_ptr(), self.K[l, p:p + n].data_ptr(),
+                                    self.V[l, p:p + n].data_ptr(), self.O[l, p:p + n].data_ptr())
+        self.graph = None
+
+    def step_direct(self):
+        kv, lib, h = self.kvc, self.kvc._lib, self.kvc._h
+        st = kv._stream()
+        kv.reset()
+        ws = kv.workspace.data_ptr()
+        cache0, blob = kv.cache.data_ptr(), kv.blob_bytes
+        for ci, (p, n) in enumerate(self.sched):
+            for l in range(self.L):
+                q, k, v, o = self.ptrs[ci, l]
+                rc = lib.kvc_prefill_chunk(h, l, q, k, v, n, p, cache0 + l * blob, ws, o, st)
+                if rc:
+                    kv._check(rc)
+
+    def step_batched(self):
+        kv = self.kvc
+        kv.reset()
+        for p, n in self.sched:
+            kv.prefill_chunk_layers(0, self.Q[:, p:p + n], self.K[:, p:p + n], self.V[:, p:p + n], p, self.O[:, p:p + n])
+
+    def capture(self):
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.step_direct()
+
+    def step_graph(self):
+        self.graph.replay()
+
+    def step_host(self, host):
+        """End-to-end: q/k/v from pinned host memory, out back to pinned host memory, every call."""
+        kv = self.kvc
+        kv.reset()
+        qh, kh, vh, oh = host
+        for p, n in self.sched:
+            for l in range(self.L):
+                kv.prefill_chunk_host(l, qh[l, p:p + n], kh[l, p:p + n], vh[l, p:p + n], p, oh[l, p:p + n])
+
+
+def time_steps(fn, steps, barrier):
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    barrier()
+    return e0.elapsed_time(e1) / 1e3, t0, t1
+
+
+def profile_pass(r: Runner, steps: int):
+    """Per-kernel CUDA-event durations (on the launching stream) and exact algorithmic work, direct calls."""
+    kv, cfg = r.kvc, r.cfg
+    work = {s: dict(bytes=0, flops=0) for s in STEPS}
+    # exact move counts need one pass with a readback after every call
+    kv.reset()
+    n_c = 0
+    for ci, (p, n) in enumerate(r.sched):
+        for l in range(r.L):
+            q, k, v, o = r.ptrs[ci, l]
+            kv._check(kv._lib.kvc_prefill_chunk(kv._h, l, q, k, v, n, p, kv.cache[l].data_ptr(), kv.workspace.data_ptr(),
+                                                o, kv._stream()))
+            moves = kv.move_counts(0).tolist() if n_c + n > cfg.budget else None
+            for s, wv in work_of_call(cfg, n, n_c, moves).items():
+                work[s]["bytes"] += wv["bytes"]; work[s]["flops"] += wv["flops"]
+        n_c = min(n_c + n, cfg.budget)
+    torch.cuda.synchronize()
+    kv.profile_enable(True)
+    for _ in range(steps):
+        r.step_direct()
+    torch.cuda.synchronize()
+    ms, cnt = kv.profile_read()
+    kv.profile_enable(False)
+    per = {}
+    for s in STEPS:
+        if cnt[s]:
+            per[s] = dict(ms_total_per_step=ms[s] / steps, launches_per_step=cnt[s] // steps,
+                          us_per_launch=1e3 * ms[s] / cnt[s], bytes_per_step=work[s]["bytes"],
+                          flops_per_step=work[s]["flops"])
+    return per
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C2", choices=sorted(CONFIGS))
+    ap.add_argument("--mode", default="graph", choices=["graph", "direct", "batched"])
+    ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (0 = all; not a headline run)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-profile", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = CONFIGS[args.workload]
+    if args.impl == "reference":
+        reference_arm(args, cfg, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    args.warmup = max(args.warmup, 3)
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    peaks = load_peaks()
+    L = args.layers if args.layers else cfg.n_layers
+    r = Runner(cfg, local_rank, L)
+    kv = r.kvc
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    step = {"direct": r.step_direct, "batched": r.step_batched, "graph": r.step_graph}[args.mode]
+    r.step_direct()                       # sets function attributes, resolves the driver entry point
+    torch.cuda.synchronize()
+    if args.mode == "graph":
+        r.capture()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert kv.status() == 0, kv.last_error()
+    launches_before = kv.launch_count()
+    if args.mode == "graph":              # a replay launches what one captured step launched
+        r.step_direct(); torch.cuda.synchronize()
+        launches_per_step = kv.launch_count() - launches_before
+    secs, t0, t1 = time_steps(step, args.steps, barrier)
+    if args.mode != "graph":
+        launches_per_step = (kv.launch_count() - launches_before) // args.steps
+    assert kv.status() == 0, kv.last_error()
+    if dist is not None:
+        t = torch.tensor([secs], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        secs = float(t.item())
+    tokens_layers = cfg.n_tokens * L
+    value = world * tokens_layers * args.steps / secs
+
+    # ---- per-kernel durations and roofline (rank 0, outside the timed region)
+    per, roof = {}, None
+    if rank == 0 and not args.no_profile:
+        per = profile_pass(r, max(3, min(args.steps, 10)))
+        ridge = peaks["tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+        for s, d in per.items():
+            sec = d["ms_total_per_step"] / 1e3
+            d["gbs"] = d["bytes_per_step"] / sec / 1e9
+            d["tflops"] = d["flops_per_step"] / sec / 1e12
+        dom = max(per, key=lambda s: per[s]["ms_total_per_step"])
+        d = per[dom]
+        ai = d["flops_per_step"] / max(d["bytes_per_step"], 1)
+        if cfg.dtype == "bf16" and dom in ("attention",) and ai > ridge:
+            roof = dict(kernel=dom, bound="tensor", achieved=d["tflops"], peak=peaks["tflops_sustained"], unit="TFLOP/s",
+                        frac=d["tflops"] / peaks["tflops_sustained"], traffic=None, peak_source=peaks["source"] + " (sustained bf16)")
+        else:
+            roof = dict(kernel=dom, bound="hbm", achieved=d["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=d["gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"])
+        roof["us_per_launch"] = d["us_per_launch"]
+        roof["arithmetic_intensity"] = ai
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        host = tuple(t.cpu().pin_memory() for t in (r.Q, r.K, r.V)) + (torch.empty(r.O.shape, dtype=r.O.dtype).pin_memory(),)
+        for _ in range(2):
+            r.step_host(host)
+        torch.cuda.synchronize()
+        e_steps = max(1, min(args.steps, 5))
+        esecs, _, _ = time_steps(lambda: r.step_host(host), e_steps, barrier)
+        if dist is not None:
+            t = torch.tensor([esecs], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            esecs = float(t.item())
+        h2d = sum(t.numel() * t.element_size() for t in host[:3])
+        d2h = host[3].numel() * host[3].element_size()
+        e2e = dict(value=world * tokens_layers * e_steps / esecs, unit=UNIT, h2d_bytes_per_step=h2d,
+                   d2h_bytes_per_step=d2h, steps=e_steps, ms_per_step=1e3 * esecs / e_steps)
+        del host
+    rows = sampler.stop()
+    clocks = sampler.summary(rows, t0, t1)
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # the same bounded sample on successive layers until about 10 s of CPU work have been spent
+        tot_dt, vals, desc, nl_done = 0.0, [], "", 0
+        while nl_done < L and tot_dt < 10.0:
+            tens = tuple(t[nl_done].double().cpu().numpy() for t in (r.Q, r.K, r.V))
+            val, dt, desc = run_oracle_sample(cfg, tens)
+            vals.append(val); tot_dt += dt; nl_done += 1
+        cpu = dict(value=len(vals) / sum(1.0 / x for x in vals), unit=UNIT, cores=cpu_threads(), kind="oracle",
+                   sample=desc.replace("layer 0", f"layers 0..{nl_done - 1}"), seconds=tot_dt)
+
+    if rank == 0:
+        logical, physical, full = kv.kv_bytes(cfg.n_tokens)
+        scale = L / cfg.n_layers
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+                "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+                           "head_dim": cfg.head_dim, "tokens": cfg.n_tokens, "block": cfg.chunk, "budget": cfg.budget,
+                           "obs_window": cfg.obs_window, "mode": args.mode, "parallelism": f"replicas x{world}",
+                           "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"},
+                "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
+                "kv_bytes": {"logical_budget": int(logical * scale), "physical_allocated": int(physical * scale),
+                             "uncompressed": int(full * scale), "blobs": kv.blob_bytes * L},
+                "kernels": per}
+        if roof:
+            line["roofline"] = roof
+        if e2e:
+            line["e2e"] = e2e
+        if cpu:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

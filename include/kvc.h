@@ -147,6 +147,10 @@ int kvc_cache_view(const kvc_ctx* ctx, int layer, void* cache, kvc_view* view);
  * a batched call). */
 int kvc_workspace_view(const kvc_ctx* ctx, void* workspace, int slot, float** lse, float** score);
 
+/* DEVICE pointer (borrowed) to the int32 [Hkv] array holding, for layer slot `slot`, how many
+ * entries the most recent eviction moved per kv-head during compaction. */
+int kvc_move_counts(const kvc_ctx* ctx, void* workspace, int slot, int** counts);
+
 /* Synchronises `stream` and returns the device status word kept in the workspace: KVC_OK, or
  * KVC_ETIMEOUT if a bounded wait inside a kernel gave up (the kernel then left early; results of
  * that call are invalid but the context and the device stay usable). */
@@ -157,6 +161,15 @@ int kvc_status(kvc_ctx* ctx, void* workspace, void* stream);
  * uncompressed uses seq_len. */
 int kvc_kv_bytes(const kvc_ctx* ctx, long long seq_len, size_t* logical, size_t* physical,
                  size_t* uncompressed);
+
+/* Per-kernel timing for measurement runs.  kvc_profile_enable(ctx, 1) makes every later call
+ * bracket each of its kernels with a pair of CUDA events on the caller's stream (host objects, no
+ * device memory).  kvc_profile_read synchronises those events and ADDS, per step index
+ * (0 append, 1 attention, 2 score, 3 select, 4 compact), the elapsed milliseconds into ms[5] and
+ * the number of launches into launches[5] (both HOST arrays), then forgets the events.
+ * Profiling perturbs end-to-end timing; leave it off in timed regions. */
+int kvc_profile_enable(kvc_ctx* ctx, int on);
+int kvc_profile_read(kvc_ctx* ctx, double* ms, long long* launches);
 
 /* Number of kernel launches the library has enqueued through this context so far. */
 long long kvc_launch_count(const kvc_ctx* ctx);

@@ -22,8 +22,8 @@ KVC_FLAG_CUDA_CORES = 1
 EXPORTS = [
     "kvc_create", "kvc_destroy", "kvc_cache_nbytes", "kvc_workspace_init", "kvc_reset",
     "kvc_prefill_chunk", "kvc_prefill_chunk_layers", "kvc_staging_nbytes", "kvc_prefill_chunk_host",
-    "kvc_cache_view", "kvc_workspace_view", "kvc_status", "kvc_kv_bytes", "kvc_launch_count",
-    "kvc_last_error",
+    "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
+    "kvc_profile_read", "kvc_launch_count", "kvc_last_error",
 ]
 
 
@@ -61,8 +61,11 @@ def load_library() -> ctypes.CDLL:
     lib.kvc_prefill_chunk_host.argtypes = [vp, i, vp, vp, vp, i, ll, vp, vp, vp, vp, vp]
     lib.kvc_cache_view.argtypes = [vp, i, vp, ctypes.POINTER(KvcView)]
     lib.kvc_workspace_view.argtypes = [vp, vp, i, ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    lib.kvc_move_counts.argtypes = [vp, vp, i, ctypes.POINTER(vp)]
     lib.kvc_status.argtypes = [vp, vp, vp]
     lib.kvc_kv_bytes.argtypes = [vp, ll, psz, psz, psz]
+    lib.kvc_profile_enable.argtypes = [vp, i]
+    lib.kvc_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.kvc_launch_count.argtypes = [vp]
     lib.kvc_launch_count.restype = ll
     lib.kvc_last_error.argtypes = [vp]
@@ -218,6 +221,13 @@ class Kvc:
         score = self.workspace[so:so + self.cfg.n_kv_heads * cap * 4].view(torch.float32)
         return lse.view(self.cfg.max_chunk, self.cfg.n_q_heads), score.view(self.cfg.n_kv_heads, cap)
 
+    def move_counts(self, slot: int = 0) -> torch.Tensor:
+        """int32 [Hkv]: entries moved per kv-head by the most recent compaction of this slot."""
+        a = ctypes.c_void_p()
+        self._check(self._lib.kvc_move_counts(self._h, self.workspace.data_ptr(), slot, ctypes.byref(a)))
+        off = a.value - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * self.cfg.n_kv_heads].view(torch.int32)
+
     def status(self) -> int:
         return self._lib.kvc_status(self._h, self.workspace.data_ptr(), self._stream())
 
@@ -225,6 +235,17 @@ class Kvc:
         a, b, c = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
         self._check(self._lib.kvc_kv_bytes(self._h, seq_len, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)))
         return a.value, b.value, c.value
+
+    def profile_enable(self, on: bool):
+        self._check(self._lib.kvc_profile_enable(self._h, int(on)))
+
+    def profile_read(self):
+        """({step: milliseconds}, {step: launches}) accumulated since profiling was enabled / last read."""
+        ms = (ctypes.c_double * 5)()
+        cnt = (ctypes.c_longlong * 5)()
+        self._check(self._lib.kvc_profile_read(self._h, ms, cnt))
+        names = ("append", "attention", "score", "select", "compact")
+        return dict(zip(names, list(ms))), dict(zip(names, list(cnt)))
 
     def launch_count(self) -> int:
         return self._lib.kvc_launch_count(self._h)

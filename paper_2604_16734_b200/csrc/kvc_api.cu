@@ -34,6 +34,9 @@ struct kvc_ctx {
   long long launches;
   EncodeTiledFn encode;
   bool use_tc;
+  bool profiling;
+  struct Prof { int kind; cudaEvent_t a, b; };
+  std::vector<Prof> prof;
   char err[512];
 };
 
@@ -97,13 +100,55 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->launches = 0;
   c->encode = nullptr;
   c->use_tc = cfg->dtype == KVC_BF16 && !(cfg->flags & KVC_FLAG_CUDA_CORES);
+  c->profiling = false;
   c->err[0] = 0;
   *out = c;
   return KVC_OK;
 }
 
+static void drop_events(kvc_ctx* c) {
+  for (auto& p : c->prof) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  c->prof.clear();
+}
+
+extern "C" int kvc_profile_enable(kvc_ctx* c, int on) {
+  if (!live(c)) return KVC_ESTATE;
+  c->profiling = on != 0;
+  if (!on) drop_events(c);
+  return KVC_OK;
+}
+
+extern "C" int kvc_profile_read(kvc_ctx* c, double* ms, long long* launches) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!ms || !launches) return KVC_EINVAL;
+  int rc = KVC_OK;
+  for (auto& p : c->prof) {
+    float t = 0.f;
+    cudaError_t e = cudaEventSynchronize(p.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&t, p.a, p.b);
+    if (e != cudaSuccess) { rc = fail(c, KVC_ECUDA, "profile event: %s", cudaGetErrorString(e)); break; }
+    ms[p.kind] += t;
+    launches[p.kind] += 1;
+  }
+  drop_events(c);
+  return rc;
+}
+
+// Brackets one kernel launch with events when profiling is on.
+struct ProfScope {
+  kvc_ctx* c; cudaStream_t st; cudaEvent_t a, b; bool on;
+  ProfScope(kvc_ctx* c_, int kind, cudaStream_t st_) : c(c_), st(st_), a(nullptr), b(nullptr), on(c_->profiling) {
+    if (!on) return;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
+    cudaEventRecord(a, st);
+    c->prof.push_back({kind, a, b});
+  }
+  ~ProfScope() { if (on) cudaEventRecord(b, st); }
+};
+
 extern "C" int kvc_destroy(kvc_ctx* c) {
   if (!live(c)) return KVC_ESTATE;
+  drop_events(c);
   c->magic = 0;
   delete c;
   return KVC_OK;
@@ -179,6 +224,13 @@ extern "C" int kvc_workspace_view(const kvc_ctx* c, void* workspace, int slot, f
   char* s = (char*)workspace + kvc::kWsHeaderBytes + (size_t)slot * c->ws_slot_bytes;
   if (lse) *lse = (float*)(s + c->lse_off);
   if (score) *score = (float*)(s + c->score_off);
+  return KVC_OK;
+}
+
+extern "C" int kvc_move_counts(const kvc_ctx* c, void* workspace, int slot, int** counts) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!workspace || !counts || slot < 0 || slot >= c->cfg.n_layers) return KVC_EINVAL;
+  *counts = (int*)((char*)workspace + kvc::kWsHeaderBytes + (size_t)slot * c->ws_slot_bytes + c->mcount_off);
   return KVC_OK;
 }
 
@@ -346,6 +398,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
 
   // a0 append
   {
+    ProfScope ps(c, 0, st);
     dim3 grid((n * g.Hkv + 7) / 8, 1, nl);
     if (f32) kvc::append_kernel<float><<<grid, 256, 0, st>>>((const float*)k, (const float*)v, (char*)cache, g);
     else kvc::append_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (char*)cache, g);
@@ -353,6 +406,8 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   }
   // a1 attention
   cudaError_t e = cudaSuccess;
+  {
+  ProfScope ps(c, 1, st);
   if (c->use_tc) {
     e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, out, ws, st) : launch_tc_attn<64>(g, tq, tk, tv, out, ws, st);
   } else if (f32) {
@@ -360,10 +415,13 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   } else {
     if (D == 128) launch_cc_attn<__nv_bfloat16, 128>(g, q, cache, out, ws, st); else launch_cc_attn<__nv_bfloat16, 64>(g, q, cache, out, ws, st);
   }
+  }
   if (e != cudaSuccess) return check_cuda(c, e, "attention launch setup");
   c->launches++;
   if (evict) {
     // a2 score
+    {
+    ProfScope ps(c, 2, st);
     if (c->use_tc) {
       e = D == 128 ? launch_tc_score<128>(g, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, tk, tqo, ws, tok_per_group, st);
     } else if (f32) {
@@ -371,14 +429,21 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     } else {
       e = D == 128 ? launch_cc_score<__nv_bfloat16, 128>(g, q, cache, ws, st) : launch_cc_score<__nv_bfloat16, 64>(g, q, cache, ws, st);
     }
+    }
     if (e != cudaSuccess) return check_cuda(c, e, "score launch setup");
     c->launches++;
     // a3 select
-    kvc::select_kernel<<<dim3(g.Hkv, 1, nl), 1024, 0, st>>>((const char*)cache, (char*)ws, g);
+    {
+      ProfScope ps(c, 3, st);
+      kvc::select_kernel<<<dim3(g.Hkv, 1, nl), 1024, 0, st>>>((const char*)cache, (char*)ws, g);
+    }
     c->launches++;
     // a4 compact: at most min(n, tot - B) entries sit at or above row B
     const int max_moves = n < g.tot - g.B ? n : g.tot - g.B;
-    kvc::compact_kernel<<<dim3((max_moves + 7) / 8, g.Hkv, nl), 256, 0, st>>>((char*)cache, (const char*)ws, g, (int)c->elem);
+    {
+      ProfScope ps(c, 4, st);
+      kvc::compact_kernel<<<dim3((max_moves + 7) / 8, g.Hkv, nl), 256, 0, st>>>((char*)cache, (const char*)ws, g, (int)c->elem);
+    }
     c->launches++;
   }
   int rc = check_cuda(c, cudaGetLastError(), "kernel launch");

@@ -310,6 +310,22 @@ static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CU
   return cudaSuccess;
 }
 template <int D>
+static cudaError_t launch_tc2_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                   void* out, void* ws, cudaStream_t st) {
+  const int smem = (2 + kvc::kStages) * (D / 64) * kvc::kSubTileBytes + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int TOK = 128 / g.G;
+  const int row_tiles = (g.n + TOK - 1) / TOK;
+  dim3 grid((row_tiles + 1) / 2, g.Hkv, g.nl);
+  kvc::attn_tc2_kernel<D><<<grid, 320, smem, st>>>(tq, tk, tv, (__nv_bfloat16*)out, (char*)ws, g);
+  return cudaSuccess;
+}
+template <int D>
 static cudaError_t launch_tc_score(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* ws,
                                    int tok_per_group, cudaStream_t st) {
   const int smem = (D / 64) * (kvc::kSubTileBytes + 256 * 128) + 1024;
@@ -408,8 +424,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   cudaError_t e = cudaSuccess;
   {
   ProfScope ps(c, 1, st);
-  if (c->use_tc) {
+  if (c->use_tc && (cf.flags & 2u)) {       // single-tile kernel kept for comparison while the pipelined one is validated
     e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, out, ws, st) : launch_tc_attn<64>(g, tq, tk, tv, out, ws, st);
+  } else if (c->use_tc) {
+    e = D == 128 ? launch_tc2_attn<128>(g, tq, tk, tv, out, ws, st) : launch_tc2_attn<64>(g, tq, tk, tv, out, ws, st);
   } else if (f32) {
     if (D == 128) launch_cc_attn<float, 128>(g, q, cache, out, ws, st); else launch_cc_attn<float, 64>(g, q, cache, out, ws, st);
   } else {

@@ -137,6 +137,32 @@ int kvc_prefill_chunk_host(kvc_ctx* ctx, int layer, const void* q_host, const vo
                            const void* v_host, int n, long long pos0, void* cache, void* workspace,
                            void* staging, void* out_host, void* stream);
 
+/* (No counterpart in the paper: an integration convenience.)
+ * kvc_prefill_chunk for callers that have no way to obtain scratch memory: code running where
+ * cudaMalloc is off limits -- inside a memory pool that owns the whole device, in a plugin that
+ * may only touch the buffers it is handed, or in a latency-critical loop where an allocation would
+ * synchronise the device.  The caller passes only the tensors it already owns (q, k, v, the layer's
+ * cache blob, out); the scratch that kvc_prefill_chunk takes as `workspace` (log-sum-exp, scores,
+ * move lists, status word) lives in a fixed array of KVC_STATIC_WS_BYTES bytes compiled into the
+ * library, which every GPU that loads the library holds until the process exits.
+ *   - The configuration must need no more than KVC_STATIC_WS_BYTES of single-layer scratch
+ *     (lse 4*Hq*max_chunk + scores 4*Hkv*cap + move lists 8*Hkv*max_chunk + ~1.5 KB); otherwise
+ *     the call returns KVC_EINVAL and kvc_last_error names both sizes.  Nothing is enqueued then.
+ *   - The first call on a device looks up the device address of the array (once per device, with
+ *     that device current); make that first call outside any stream capture.
+ *   - The array is shared by every context and every call on the device and keeps what the last
+ *     call left there; the call clears the status word it needs zeroed.  Two calls whose GPU work
+ *     overlaps (different streams, or different threads without ordering) race on it: keep all
+ *     users of this entry point on one stream, or order them with events.
+ *   - Calls cudaMalloc/cudaFree never, and returns KVC_ESTATE while kvc_profile_enable is on
+ *     (profiling creates events).
+ * Arguments and results are otherwise exactly those of kvc_prefill_chunk.  kvc_status_static reads
+ * the status word of the current device's array after synchronising `stream`. */
+#define KVC_STATIC_WS_BYTES (1u << 20)
+int kvc_prefill_chunk_static(kvc_ctx* ctx, int layer, const void* q, const void* k, const void* v,
+                             int n, long long pos0, void* cache, void* out, void* stream);
+int kvc_status_static(kvc_ctx* ctx, void* stream);
+
 /* Output of Alg. 1: the compressed cache of one layer, as borrowed pointers. */
 int kvc_cache_view(const kvc_ctx* ctx, int layer, void* cache, kvc_view* view);
 

@@ -22,6 +22,7 @@ KVC_FLAG_CUDA_CORES = 1
 EXPORTS = [
     "kvc_create", "kvc_destroy", "kvc_cache_nbytes", "kvc_workspace_init", "kvc_reset",
     "kvc_prefill_chunk", "kvc_prefill_chunk_layers", "kvc_staging_nbytes", "kvc_prefill_chunk_host",
+    "kvc_prefill_chunk_static", "kvc_status_static",
     "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
     "kvc_profile_read", "kvc_launch_count", "kvc_last_error",
 ]
@@ -59,6 +60,8 @@ def load_library() -> ctypes.CDLL:
     lib.kvc_prefill_chunk_layers.argtypes = [vp, i, i, vp, ll, vp, vp, ll, i, ll, vp, sz, vp, vp, ll, vp]
     lib.kvc_staging_nbytes.argtypes = [vp, psz]
     lib.kvc_prefill_chunk_host.argtypes = [vp, i, vp, vp, vp, i, ll, vp, vp, vp, vp, vp]
+    lib.kvc_prefill_chunk_static.argtypes = [vp, i, vp, vp, vp, i, ll, vp, vp, vp]
+    lib.kvc_status_static.argtypes = [vp, vp]
     lib.kvc_cache_view.argtypes = [vp, i, vp, ctypes.POINTER(KvcView)]
     lib.kvc_workspace_view.argtypes = [vp, vp, i, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.kvc_move_counts.argtypes = [vp, vp, i, ctypes.POINTER(vp)]
@@ -192,6 +195,20 @@ class Kvc:
                                                      self.cache[layer].data_ptr(), self.workspace.data_ptr(),
                                                      self.staging.data_ptr(), _ptr(out), self._stream()))
         return out
+
+    def prefill_chunk_static(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, pos0: int,
+                             out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """prefill_chunk with the library's built-in scratch array instead of ``self.workspace``:
+        for callers that cannot allocate device memory.  One stream at a time per device."""
+        if out is None:
+            out = torch.empty_like(q)
+        assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and out.is_contiguous()
+        self._check(self._lib.kvc_prefill_chunk_static(self._h, layer, _ptr(q), _ptr(k), _ptr(v), q.shape[0], pos0,
+                                                       self.cache[layer].data_ptr(), _ptr(out), self._stream()))
+        return out
+
+    def status_static(self) -> int:
+        return self._lib.kvc_status_static(self._h, self._stream())
 
     def cache_view(self, layer: int) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor, int]:
         """(K [Hkv][cap][d], V [Hkv][cap][d], pos [Hkv][cap], len): tensors alias the cache blob."""

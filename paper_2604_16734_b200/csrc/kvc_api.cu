@@ -517,3 +517,52 @@ extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host,
   if (rc) return rc;
   return check_cuda(c, cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st), "D2H out");
 }
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant: the scratch area is a fixed device array compiled into the library.
+// In host code `g_static_ws` is only a handle for the runtime, not a device address; the address
+// each device gives it is looked up once per device and cached here.
+static __device__ __align__(256) unsigned char g_static_ws[KVC_STATIC_WS_BYTES];
+static const int kMaxDevices = 64;
+static void* g_static_ws_ptr[kMaxDevices] = {nullptr};
+
+static int static_ws_for_current_device(kvc_ctx* c, void** ptr) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return check_cuda(c, e, "cudaGetDevice");
+  if (dev < 0 || dev >= kMaxDevices) return fail(c, KVC_EINVAL, "device ordinal %d not supported by the static scratch", dev);
+  if (dev != c->cfg.device) return fail(c, KVC_ESTATE, "current CUDA device %d is not the context's device %d", dev, c->cfg.device);
+  if (!g_static_ws_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_ws);
+    if (e != cudaSuccess || !p) return check_cuda(c, e == cudaSuccess ? cudaErrorInvalidSymbol : e, "cudaGetSymbolAddress(static scratch)");
+    g_static_ws_ptr[dev] = p;
+  }
+  *ptr = g_static_ws_ptr[dev];
+  return KVC_OK;
+}
+
+extern "C" int kvc_prefill_chunk_static(kvc_ctx* c, int layer, const void* q, const void* k, const void* v, int n,
+                                        long long pos0, void* cache, void* out, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (c->profiling) return fail(c, KVC_ESTATE, "kvc_prefill_chunk_static needs profiling off");
+  const size_t need = kvc::kWsHeaderBytes + c->ws_slot_bytes;          // header + one layer slot
+  if (need > (size_t)KVC_STATIC_WS_BYTES)
+    return fail(c, KVC_EINVAL, "configuration needs %zu bytes of scratch, the built-in scratch holds %u", need,
+                (unsigned)KVC_STATIC_WS_BYTES);
+  void* ws = nullptr;
+  int rc = static_ws_for_current_device(c, &ws);
+  if (rc) return rc;
+  // the array keeps the previous call's contents: only the status word has to start at zero
+  rc = check_cuda(c, cudaMemsetAsync(ws, 0, kvc::kWsHeaderBytes, (cudaStream_t)stream), "cudaMemsetAsync(static scratch)");
+  if (rc) return rc;
+  return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, ws, out, 0, (cudaStream_t)stream);
+}
+
+extern "C" int kvc_status_static(kvc_ctx* c, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  void* ws = nullptr;
+  int rc = static_ws_for_current_device(c, &ws);
+  if (rc) return rc;
+  return kvc_status(c, ws, stream);
+}

@@ -442,7 +442,6 @@ def main():
 
     if rank == 0:
         logical, physical, full = kv.kv_bytes(cfg.n_tokens)
-        scale = L / cfg.n_layers
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
@@ -451,8 +450,8 @@ def main():
                            "obs_window": cfg.obs_window, "mode": args.mode, "parallelism": f"replicas x{world}",
                            "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"},
                 "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
-                "kv_bytes": {"logical_budget": int(logical * scale), "physical_allocated": int(physical * scale),
-                             "uncompressed": int(full * scale), "blobs": kv.blob_bytes * L},
+                "kv_bytes": {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,
+                             "blobs_incl_positions": kv.blob_bytes * L},
                 "kernels": per}
         if roof:
             line["roofline"] = roof

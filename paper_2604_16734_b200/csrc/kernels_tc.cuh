@@ -392,9 +392,16 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
         for (int c = 0; c < 128; ++c)
           if (c >= lim) sr[c] = 0xff800000u;                  // -inf
       }
-      float mx = -INFINITY;
+      float mx4[8];                                           // independent chains: latency, not issue, is the cost
 #pragma unroll
-      for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+      for (int i = 0; i < 8; ++i) mx4[i] = __uint_as_float(sr[i]);
+#pragma unroll
+      for (int c = 8; c < 128; c += 8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sr[c + i]));
+      }
+      const float mx = fmaxf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])),
+                             fmaxf(fmaxf(mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
       const float m_new = mx * p.scale_log2;                  // scale > 0
       if (j == 0) {
         m_ref = m_new == -INFINITY ? 0.f : m_new;
@@ -418,7 +425,7 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
         }
       }
       const float neg_m = -m_ref;
-      float psum = 0.f;
+      float ps[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t pk[16];
@@ -426,12 +433,13 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
         for (int i = 0; i < 16; ++i) {
           const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i]), p.scale_log2, neg_m));
           const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
-          psum += p0 + p1;
+          ps[(i & 1) * 2] += p0;
+          ps[(i & 1) * 2 + 1] += p1;
           pk[i] = pack_bf16x2(p0, p1);
         }
         tmem_st16(tmem_S + c * 16, pk);
       }
-      l += psum;
+      l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(&sh.p_full[t]);

@@ -210,7 +210,7 @@ def reference_arm(args, cfg, rank):
 # our arm
 
 class Runner:
-    def __init__(self, cfg, device_index, n_layers=None):
+    def __init__(self, cfg, device_index, n_layers=None, flags=0):
         from paper_2604_16734_b200.binding import Kvc
         self.cfg = cfg
         self.L = cfg.n_layers if n_layers is None else n_layers
@@ -226,7 +226,7 @@ class Runner:
         del wl
         self.O = torch.empty_like(self.Q)
         self.kvc = Kvc(self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk,
-                       cfg.obs_window, device=device_index)
+                       cfg.obs_window, device=device_index, flags=flags)
         self.sched = cfg.chunks()
         # raw pointers of every (block, layer) slice, so the per-call host work is one ctypes call
         self.ptrs = {}
@@ -329,6 +329,7 @@ def main():
     ap.add_argument("--workload", default="C2", choices=sorted(CONFIGS))
     ap.add_argument("--mode", default="graph", choices=["graph", "direct", "batched"])
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (0 = all; not a headline run)")
+    ap.add_argument("--flags", type=int, default=0, help="KVC_FLAG_* bits passed to kvc_create (kernel selection, diagnostics)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
@@ -357,7 +358,7 @@ def main():
 
     peaks = load_peaks()
     L = args.layers if args.layers else cfg.n_layers
-    r = Runner(cfg, local_rank, L)
+    r = Runner(cfg, local_rank, L, args.flags)
     kv = r.kvc
     sampler = ClockSampler(local_rank)
     sampler.start()

@@ -24,6 +24,7 @@ struct Geom {
   long long lse_off, score_off, msrc_off, mdst_off, mcount_off;   // byte offsets inside a slot
 };
 
+static constexpr int kNumSMs = 148;          // B200
 static constexpr int kWsHeaderBytes = 256;   // status word lives at byte 0 of the workspace
 
 __device__ __forceinline__ char* ws_slot(char* ws, const Geom& p, int slot) {

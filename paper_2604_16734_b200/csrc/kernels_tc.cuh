@@ -15,196 +15,6 @@ static constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 bf16 (one 128
 // with the tokens, row r = (token - tok0) * G + (head - g*G), so keys and values are read once per
 // kv-head.  A tile holds TOK = 128 / G tokens (TOK * G <= 128 rows).
 
-struct TcSmemAttn {
-  uint64_t bar_q, bar_kv, bar_s, bar_p, bar_o;
-  uint32_t tmem_base;
-  int abort_flag;
-};
-
-// ------------------------------------------------------------------------------------------------
-// a1 attention, one 128-row tile per CTA.
-// Warps 0-3: softmax (thread = one row = one TMEM lane).  Warp 4: one elected lane issues the TMA
-// loads and the MMAs.  Per 128-key tile: S = Q K^T (tcgen05, fp32 in TMEM) -> online softmax in
-// registers -> P (bf16) written back to TMEM over S -> O += P V (A operand from TMEM, V read
-// MN-major from shared memory).
-// grid (ceil(n / TOK), Hkv, nl), block 160, dynamic smem 3 * (D/64) * 16 KB + 1 KB alignment slack.
-template <int D>
-__global__ void __launch_bounds__(160) attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
-                                                      const __grid_constant__ CUtensorMap tm_k,
-                                                      const __grid_constant__ CUtensorMap tm_v,
-                                                      __nv_bfloat16* __restrict__ out, char* __restrict__ ws, Geom p) {
-  constexpr int NSUB = D / 64;
-  constexpr uint32_t TMEM_COLS = 256;          // S/P at columns [0,128), O at [128, 128 + D)
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;
-  uint8_t* sK = sQ + NSUB * kSubTileBytes;
-  uint8_t* sV = sK + NSUB * kSubTileBytes;
-  __shared__ TcSmemAttn sh;
-
-  const int layer = blockIdx.z, g = blockIdx.y;
-  const int TOK = 128 / p.G, rows = TOK * p.G;
-  const int tok0 = blockIdx.x * TOK;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int last_tok = min(tok0 + TOK, p.n) - 1;
-  const int kv_end = p.n_c + last_tok + 1;
-  const int n_tiles = (kv_end + 127) / 128;
-
-  if (threadIdx.x == 0) {
-    mbar_init(&sh.bar_q, 1); mbar_init(&sh.bar_kv, 1); mbar_init(&sh.bar_s, 1);
-    mbar_init(&sh.bar_p, 128); mbar_init(&sh.bar_o, 1);
-    sh.abort_flag = 0;
-    mbar_fence_init();
-  }
-  // rows of the Q tile that TMA never writes (rows >= TOK*G) must still be finite
-  for (int i = threadIdx.x; i < NSUB * (128 - rows) * 8; i += blockDim.x) {
-    const int sub = i / ((128 - rows) * 8), rem = i % ((128 - rows) * 8);
-    reinterpret_cast<uint4*>(sQ + sub * kSubTileBytes + rows * 128)[rem] = make_uint4(0, 0, 0, 0);
-  }
-  fence_proxy_async_smem();
-  if (warp == 4) {
-    tmem_alloc(&sh.tmem_base, TMEM_COLS);
-    tmem_relinquish();
-  }
-  tc_fence_before_sync();
-  __syncthreads();
-  tc_fence_after_sync();
-  const uint32_t tmem = sh.tmem_base;
-  const uint32_t tmem_S = tmem, tmem_O = tmem + 128;
-  volatile int* abort_flag = &sh.abort_flag;
-
-  if (warp == 4) {
-    if (lane == 0) {
-      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
-      mbar_expect_tx(&sh.bar_q, NSUB * rows * 128);
-      for (int sub = 0; sub < NSUB; ++sub)
-        tma_load_4d(sQ + sub * kSubTileBytes, &tm_q, &sh.bar_q, sub * 64, g * p.G, tok0, layer);
-      const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
-      const uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
-      const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
-      bool ok = true;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        if (j > 0) ok = mbar_wait(&sh.bar_o, (j - 1) & 1, abort_flag);     // K/V smem and S/P TMEM free again
-        if (!ok) break;
-        mbar_expect_tx(&sh.bar_kv, 2 * NSUB * kSubTileBytes);
-        for (int sub = 0; sub < NSUB; ++sub) {
-          tma_load_4d(sK + sub * kSubTileBytes, &tm_k, &sh.bar_kv, sub * 64, j * 128, g, layer);
-          tma_load_4d(sV + sub * kSubTileBytes, &tm_v, &sh.bar_kv, sub * 64, j * 128, g, layer);
-        }
-        if (j == 0) ok = mbar_wait(&sh.bar_q, 0, abort_flag);
-        ok = ok && mbar_wait(&sh.bar_kv, j & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {                 // S = Q K^T, 16 of the d columns per MMA
-          const uint32_t off = (kk / 4) * kSubTileBytes + (kk % 4) * 32;
-          mma_ss(tmem_S, smem_desc_sw128(aQ + off, 16, 1024), smem_desc_sw128(aK + off, 16, 1024), idesc_qk,
-                 kk > 0);
-        }
-        mma_commit(&sh.bar_s);
-        ok = mbar_wait(&sh.bar_p, j & 1, abort_flag);         // P is in TMEM
-        if (!ok) break;
-        tc_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)                        // O += P V, 16 keys per MMA
-          mma_ts(tmem_O, tmem_S + kk * 8, smem_desc_sw128(aV + kk * 2048, kSubTileBytes, 1024), idesc_pv,
-                 (j > 0 || kk > 0));
-        mma_commit(&sh.bar_o);
-      }
-    }
-    __syncwarp();
-  } else {
-    const int r = threadIdx.x;                                // row of the tile = TMEM lane
-    const int tok = tok0 + r / p.G, hh = r % p.G;
-    const bool row_valid = r < rows && tok < p.n;
-    const int limit = p.n_c + tok + 1;                        // keys [0, limit) are visible to this row
-    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
-    float m = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
-      ok = mbar_wait(&sh.bar_s, j & 1, abort_flag);
-      if (!ok) break;
-      tc_fence_after_sync();
-      uint32_t sr[128];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tmem_S + lane_addr + c * 32, sr + c * 32);
-      tmem_wait_ld();
-      const int lim = limit - j * 128;                        // columns [0, lim) of this tile are visible
-      float tmax = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 128; ++c) {
-        float t = __uint_as_float(sr[c]) * p.scale_log2;
-        t = c < lim ? t : -INFINITY;
-        sr[c] = __float_as_uint(t);
-        tmax = fmaxf(tmax, t);
-      }
-      const float m_new = fmaxf(m, tmax);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;   // fully masked so far: every p is 0
-      const float corr = fast_exp2(m - m_use);
-      float psum = 0.f;
-      uint32_t pk[64];
-#pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        const float p0 = fast_exp2(__uint_as_float(sr[2 * c]) - m_use);
-        const float p1 = fast_exp2(__uint_as_float(sr[2 * c + 1]) - m_use);
-        psum += p0 + p1;
-        pk[c] = pack_bf16x2(p0, p1);
-      }
-      l = l * corr + psum;
-      m = m_new;
-      if (j > 0) {                                            // rescale the running output
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tmem_O + lane_addr + c * 32, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
-          tmem_st32(tmem_O + lane_addr + c * 32, o);
-        }
-      }
-      tmem_st32(tmem_S + lane_addr, pk);
-      tmem_st32(tmem_S + lane_addr + 32, pk + 32);
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(&sh.bar_p);
-    }
-    if (ok) ok = mbar_wait(&sh.bar_o, (n_tiles - 1) & 1, abort_flag);
-    if (ok) {
-      tc_fence_after_sync();
-      const float inv = 1.f / l;
-      __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tmem_O + lane_addr + c * 32, o);
-        tmem_wait_ld();
-        if (row_valid) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 vv;
-            vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-            vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-            vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-            vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-            reinterpret_cast<uint4*>(orow + c * 32)[i] = vv;
-          }
-        }
-      }
-      if (row_valid) {
-        float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
-        lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m + log2f(l)) * 0.6931471805599453f;
-      }
-    }
-  }
-  tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 4) {
-    tc_fence_after_sync();
-    tmem_dealloc(tmem, TMEM_COLS);
-  }
-  if (threadIdx.x == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
-}
 
 // ------------------------------------------------------------------------------------------------
 // a1 attention, two 128-row tiles (A, B) per CTA, software pipelined.
@@ -471,6 +281,390 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
         lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_ref + log2f(l)) * 0.6931471805599453f;
       }
     }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+}
+
+// ------------------------------------------------------------------------------------------------
+// a1 attention (Eq. 1): two 128-row tiles (A, B) per CTA, software pipelined, with the key range
+// optionally split over the CTAs of a thread-block cluster.
+//   warps 0-3   softmax of tile A     (thread = one row = one TMEM lane), 216 registers
+//   warps 4-7   softmax of tile B
+//   warp  8     TMA producer: Q tiles once, then K_j, V_j, K_j+1, ... through a ring of kStages 32 KB slots
+//   warp  9     MMA issuer.  Per key tile j:  O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ; O_B += P_B V_j ;
+//               S_B = Q_B K_{j+1}^T, so the tensor pipe works on one row tile while the CUDA cores run
+//               the softmax of the other.  P is handed over in two halves (64 keys each) so the first
+//               PV MMAs start while the second half of the exponentials is still being computed.
+//   warps 10-11 only give their registers away (setmaxnreg works on groups of four warps)
+// TMEM columns: S_A/P_A [0,128)  S_B/P_B [128,256)  O_A [256,384)  O_B [384,512).
+// The running output is rescaled lazily: a row keeps its reference maximum until the true maximum
+// has grown by more than 2^8, so P stays below 256 and O rarely needs touching.
+//
+// Key split: with cluster size S the CTA of cluster rank s handles key tiles [s*T/S, (s+1)*T/S) of
+// its row-tile pair and ends with a partial (O, m, l).  The partials are exchanged through
+// distributed shared memory: every CTA parks its O tiles (fp32, column-major so that lanes write
+// consecutive words) in its own ring buffer, the cluster synchronises, and rank s combines and
+// writes rows [s*128/S, (s+1)*128/S) of both tiles.  Nothing but the final result goes to HBM.
+// grid (ceil(ceil(n/TOK)/2) * S, Hkv, nl), cluster (S,1,1), block 384,
+// dynamic smem (2 + kStages) * (D/64) * 16 KB + 1 KB.
+static constexpr int kAttnThreads = 384;
+
+struct TcSmemAttn3 {
+  uint64_t q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_half[2][2], pv_done[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  float stat_m[2][128], stat_l[2][128];   // per row: reference maximum (log2 units, -inf if the row saw no key) and sum
+};
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                                   const __grid_constant__ CUtensorMap tm_k,
+                                                                   const __grid_constant__ CUtensorMap tm_v,
+                                                                   __nv_bfloat16* __restrict__ out,
+                                                                   char* __restrict__ ws, Geom p, int S) {
+  constexpr int NSUB = D / 64;
+  constexpr int TILE_BYTES = NSUB * kSubTileBytes;
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr float kRescaleThreshold = 8.f;      // log2 units
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;                            // two tiles
+  uint8_t* ring = smem + 2 * TILE_BYTES;         // kStages tiles; after the key loop: the parked O tiles
+  __shared__ TcSmemAttn3 sh;
+
+  const int layer = blockIdx.z, g = blockIdx.y;
+  const int split = S > 1 ? static_cast<int>(cluster_ctarank()) : 0;
+  const int pair = blockIdx.x / S;
+  const int TOK = 128 / p.G, rows = TOK * p.G;
+  const int tokA = pair * 2 * TOK, tokB = tokA + TOK;
+  const bool has_B = tokB < p.n;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int last_tok = min(tokA + 2 * TOK, p.n) - 1;
+  const int kv_end = p.n_c + last_tok + 1;
+  const int T = (kv_end + 127) / 128;            // key tiles this pair of row tiles can see
+  const int t_begin = split * T / S, t_end = (split + 1) * T / S;
+  const int Tl = t_end - t_begin;                // key tiles of this CTA (0 is possible when S > T)
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sh.q_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.pv_done[i], 1);
+      mbar_init(&sh.p_half[i][0], 128); mbar_init(&sh.p_half[i][1], 128);
+    }
+    for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
+    sh.abort_flag = 0;
+    mbar_fence_init();
+  }
+  // rows of the Q tiles that TMA never writes (rows >= TOK*G) must still be finite
+  {
+    const int pad16 = (128 - rows) * 8;          // 16-byte units per sub-tile
+    for (int i = threadIdx.x; i < 2 * NSUB * pad16; i += blockDim.x) {
+      const int sub = i / pad16, rem = i % pad16;
+      reinterpret_cast<uint4*>(sQ + sub * kSubTileBytes + rows * 128)[rem] = make_uint4(0, 0, 0, 0);
+    }
+  }
+  fence_proxy_async_smem();
+  if (warp == 8) {
+    tmem_alloc(&sh.tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sh.tmem_base;
+  volatile int* abort_flag = &sh.abort_flag;
+
+  if (warp >= 8) {
+    reg_dec<72>();
+    if (warp == 8) {
+      // ---------------------------------------------------------------- TMA producer
+      if (lane == 0) {
+        tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
+        pdl_wait();                                // the block's keys were appended by the previous kernel
+      }
+      if (lane == 0 && Tl > 0) {
+        mbar_expect_tx(&sh.q_full[0], NSUB * rows * 128);
+        for (int sub = 0; sub < NSUB; ++sub)
+          tma_load_4d(sQ + sub * kSubTileBytes, &tm_q, &sh.q_full[0], sub * 64, g * p.G, tokA, layer);
+        if (has_B) {
+          mbar_expect_tx(&sh.q_full[1], NSUB * rows * 128);
+          for (int sub = 0; sub < NSUB; ++sub)
+            tma_load_4d(sQ + TILE_BYTES + sub * kSubTileBytes, &tm_q, &sh.q_full[1], sub * 64, g * p.G, tokB, layer);
+        }
+        for (int i = 0; i < 2 * Tl; ++i) {         // item 2j = K of tile t_begin + j, item 2j+1 = V of it
+          const int slot = i % kStages, round = i / kStages;
+          if (round > 0 && !mbar_wait(&sh.kv_empty[slot], (round - 1) & 1, abort_flag)) break;
+          mbar_expect_tx(&sh.kv_full[slot], TILE_BYTES);
+          const CUtensorMap* tm = (i & 1) ? &tm_v : &tm_k;
+          for (int sub = 0; sub < NSUB; ++sub)
+            tma_load_4d(ring + slot * TILE_BYTES + sub * kSubTileBytes, tm, &sh.kv_full[slot], sub * 64,
+                        (t_begin + (i >> 1)) * 128, g, layer);
+        }
+      }
+    } else if (warp == 9) {
+      // ---------------------------------------------------------------- MMA issuer
+      if (lane == 0 && Tl > 0) {
+        const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
+        const uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
+        const uint32_t aQ = smem_u32(sQ), aR = smem_u32(ring);
+        auto issue_S = [&](int t, int slot) {      // S_t = Q_t K^T, 16 of the d columns per MMA
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk / 4) * kSubTileBytes + (kk % 4) * 32;
+            mma_ss(tmem + t * 128, smem_desc_sw128(aQ + t * TILE_BYTES + off, 16, 1024),
+                   smem_desc_sw128(aR + slot * TILE_BYTES + off, 16, 1024), idesc_qk, kk > 0);
+          }
+        };
+        auto issue_PV = [&](int t, int slot, int half, bool acc) {   // O_t += P_t V, 16 keys per MMA, 64 keys per half
+#pragma unroll
+          for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
+            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
+                   smem_desc_sw128(aR + slot * TILE_BYTES + kk * 2048, kSubTileBytes, 1024), idesc_pv, acc || kk > 0);
+        };
+        bool ok = mbar_wait(&sh.q_full[0], 0, abort_flag) && mbar_wait(&sh.kv_full[0], 0, abort_flag);
+        if (ok) {
+          tc_fence_after_sync();
+          issue_S(0, 0);
+          mma_commit(&sh.s_full[0]);
+          if (has_B) {
+            ok = mbar_wait(&sh.q_full[1], 0, abort_flag);
+            if (ok) { issue_S(1, 0); mma_commit(&sh.s_full[1]); }
+          }
+          mma_commit(&sh.kv_empty[0]);
+        }
+        for (int j = 0; j < Tl && ok; ++j) {
+          const int iv = 2 * j + 1, ik = 2 * j + 2;
+          const int slotV = iv % kStages, slotK = ik % kStages;
+          const bool more = j + 1 < Tl;
+          for (int t = 0; t < (has_B ? 2 : 1) && ok; ++t) {
+            ok = mbar_wait(&sh.p_half[t][0], j & 1, abort_flag);
+            if (ok && t == 0) ok = mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            issue_PV(t, slotV, 0, j > 0);
+            ok = mbar_wait(&sh.p_half[t][1], j & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            issue_PV(t, slotV, 1, true);
+            mma_commit(&sh.pv_done[t]);
+            if (more) {
+              if (t == 0) {
+                ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+              }
+              issue_S(t, slotK);
+              mma_commit(&sh.s_full[t]);
+            }
+          }
+          if (!ok) break;
+          mma_commit(&sh.kv_empty[slotV]);
+          if (more) mma_commit(&sh.kv_empty[slotK]);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    reg_inc<216>();
+    // ---------------------------------------------------------------- softmax + epilogue of tile t
+    const int t = warp >> 2;
+    const int r = (warp & 3) * 32 + lane;                     // row of the tile = TMEM lane
+    const int tok0 = t ? tokB : tokA;
+    const int tok = tok0 + r / p.G, hh = r % p.G;
+    const bool row_valid = r < rows && tok < p.n;
+    const int limit = p.n_c + tok + 1;                        // keys [0, limit) are visible to this row
+    const int tile_min_limit = p.n_c + tok0 + 1;              // smallest limit of any row of the tile
+    const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t tmem_S = tmem + t * 128 + lane_addr, tmem_O = tmem + 256 + t * 128 + lane_addr;
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    const bool active = t == 0 || has_B;
+    if (active) {
+      for (int j = 0; j < Tl; ++j) {
+        const int kt = t_begin + j;                           // key tile index
+        ok = mbar_wait(&sh.s_full[t], j & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t sr[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(tmem_S + c * 32, sr + c * 32);
+        tmem_wait_ld();
+        if ((kt + 1) * 128 > tile_min_limit) {                // diagonal or tail tile: mask
+          const int lim = limit - kt * 128;
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (c >= lim) sr[c] = 0xff800000u;                // -inf
+        }
+        float mx4[8];                                         // independent chains: latency, not issue, is the cost
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mx4[i] = __uint_as_float(sr[i]);
+#pragma unroll
+        for (int c = 8; c < 128; c += 8) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sr[c + i]));
+        }
+        const float mx = fmaxf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])),
+                               fmaxf(fmaxf(mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
+        const float m_new = mx * p.scale_log2;                // scale > 0
+        if (j == 0) {
+          m_ref = m_new == -INFINITY ? 0.f : m_new;
+        } else {
+          const bool grow = m_new > m_ref + kRescaleThreshold;
+          if (__any_sync(0xffffffffu, grow)) {
+            const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;
+            if (grow) { m_ref = m_new; l *= f; }
+            ok = mbar_wait(&sh.pv_done[t], (j - 1) & 1, abort_flag);   // O_t holds every earlier tile
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[32];
+              tmem_ld32(tmem_O + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+              tmem_st32(tmem_O + c * 32, o);
+            }
+          }
+        }
+        const float neg_m = -m_ref;
+        float ps[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i]), p.scale_log2, neg_m));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
+            ps[(i & 1) * 2] += p0;
+            ps[(i & 1) * 2 + 1] += p1;
+            pk[i] = pack_bf16x2(p0, p1);
+          }
+          tmem_st16(tmem_S + c * 16, pk);
+          if (c & 1) {                                        // 64 keys of P are in TMEM: release them to the MMA warp
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&sh.p_half[t][c >> 1]);
+          }
+        }
+        l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
+      }
+      if (ok && Tl > 0) ok = mbar_wait(&sh.pv_done[t], (Tl - 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);                       // the TMEM accesses below are warp-wide
+      if (ok && Tl > 0) tc_fence_after_sync();
+      if (S == 1) {
+        if (ok) {
+          const float inv = 1.f / l;
+          __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D;
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_O + c * 32, o);
+            tmem_wait_ld();
+            if (row_valid) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                uint4 vv;
+                vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+                vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+                vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+                vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+                reinterpret_cast<uint4*>(orow + c * 32)[i] = vv;
+              }
+            }
+          }
+          if (row_valid) {
+            float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
+            lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_ref + log2f(l)) * 0.6931471805599453f;
+          }
+        }
+      } else {
+        // park this CTA's partial of tile t: O column-major [D][128] fp32 in the ring, m and l beside the barriers.
+        // Every MMA of the CTA (both tiles) has to be complete before the ring is overwritten.
+        if (has_B) named_barrier(1, 256);
+        float* stg = reinterpret_cast<float*>(ring) + t * (D * 128);
+        if (ok && Tl > 0) {
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_O + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) stg[(c * 32 + i) * 128 + r] = __uint_as_float(o[i]);
+          }
+        }
+        sh.stat_m[t][r] = (ok && l > 0.f) ? m_ref : -INFINITY;
+        sh.stat_l[t][r] = l;
+      }
+    }
+  }
+
+  if (S > 1) {
+    cluster_arrive();                                         // partials of every rank are in place
+    cluster_wait();
+    if (warp < 8) {
+      // rank `split` combines rows [r0, r1) of both tiles: O = sum_s 2^(m_s - m*) O_s / sum_s 2^(m_s - m*) l_s
+      const int rows_per = (128 + S - 1) / S;
+      const int r0 = min(128, split * rows_per), r1 = min(128, r0 + rows_per), nrows = r1 - r0;
+      const int per_tile = nrows * (D / 32);                  // work items: (row, group of 32 columns)
+      const uint32_t a_stg = smem_u32(ring), a_m = smem_u32(&sh.stat_m[0][0]), a_l = smem_u32(&sh.stat_l[0][0]);
+      for (int item = threadIdx.x; item < (has_B ? 2 : 1) * per_tile; item += 256) {
+        const int t = item / per_tile, rem = item % per_tile;
+        const int r = r0 + rem % nrows, cg = rem / nrows;
+        const int tok = (t ? tokB : tokA) + r / p.G, hh = r % p.G;
+        if (!(r < rows && tok < p.n)) continue;
+        float ms[8], wt[8];
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+          ms[s] = -INFINITY;
+          if (s < S) ms[s] = dsmem_ld_f32(dsmem_addr(a_m + (t * 128 + r) * 4, s));
+          m_all = fmaxf(m_all, ms[s]);
+        }
+        float L = 0.f;
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+          wt[s] = 0.f;
+          if (s < S && ms[s] != -INFINITY) {
+            wt[s] = fast_exp2(ms[s] - m_all);
+            L = fmaf(wt[s], dsmem_ld_f32(dsmem_addr(a_l + (t * 128 + r) * 4, s)), L);
+          }
+        }
+        float acc[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+          if (s < S && wt[s] != 0.f) {
+            const uint32_t a = dsmem_addr(a_stg + ((t * D + cg * 32) * 128 + r) * 4, s);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = fmaf(wt[s], dsmem_ld_f32(a + i * 512), acc[i]);
+          }
+        }
+        const float inv = 1.f / L;
+        __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D + cg * 32;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint4 vv;
+          vv.x = pack_bf16x2(acc[8 * i + 0] * inv, acc[8 * i + 1] * inv);
+          vv.y = pack_bf16x2(acc[8 * i + 2] * inv, acc[8 * i + 3] * inv);
+          vv.z = pack_bf16x2(acc[8 * i + 4] * inv, acc[8 * i + 5] * inv);
+          vv.w = pack_bf16x2(acc[8 * i + 6] * inv, acc[8 * i + 7] * inv);
+          reinterpret_cast<uint4*>(orow)[i] = vv;
+        }
+        if (cg == 0) {
+          float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
+          lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_all + log2f(L)) * 0.6931471805599453f;
+        }
+      }
+    }
+    cluster_arrive();                                         // nobody leaves while its shared memory is being read
+    cluster_wait();
   }
   tc_fence_before_sync();
   __syncthreads();

@@ -294,20 +294,43 @@ static cudaError_t launch_cc_score(const Geom& g, const void* q, void* cache, vo
   return cudaSuccess;
 }
 
+// Number of CTAs the key range of one row-tile pair is split over (= cluster size): enough to put
+// a CTA on every SM when the row tiles alone cannot, never more than the key tiles available.
+static int attn_key_splits(const Geom& g) {
+  const int TOK = 128 / g.G;
+  const int pairs = ((g.n + TOK - 1) / TOK + 1) / 2;
+  const long long base = (long long)pairs * g.Hkv * g.nl;
+  const int T = (g.tot + 127) / 128;
+  int S = (int)(kvc::kNumSMs / base);
+  if (S > 8) S = 8;                    // portable cluster size limit
+  if (S > T) S = T;
+  return S < 1 ? 1 : S;
+}
+
 template <int D>
-static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                  void* out, void* ws, cudaStream_t st) {
-  const int smem = 3 * (D / 64) * kvc::kSubTileBytes + 1024;
+static cudaError_t launch_tc3_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                   void* out, void* ws, int S, cudaStream_t st) {
+  const int smem = (2 + kvc::kStages) * (D / 64) * kvc::kSubTileBytes + 1024;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc3_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const int TOK = 128 / g.G;
-  dim3 grid((g.n + TOK - 1) / TOK, g.Hkv, g.nl);
-  kvc::attn_tc_kernel<D><<<grid, 160, smem, st>>>(tq, tk, tv, (__nv_bfloat16*)out, (char*)ws, g);
-  return cudaSuccess;
+  const int pairs = ((g.n + TOK - 1) / TOK + 1) / 2;
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  lc.gridDim = dim3(pairs * S, g.Hkv, g.nl);
+  lc.blockDim = dim3(kvc::kAttnThreads, 1, 1);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = S; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kvc::attn_tc3_kernel<D>, tq, tk, tv, (__nv_bfloat16*)out, (char*)ws, g, S);
 }
 template <int D>
 static cudaError_t launch_tc2_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
@@ -424,10 +447,11 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   cudaError_t e = cudaSuccess;
   {
   ProfScope ps(c, 1, st);
-  if (c->use_tc && (cf.flags & 2u)) {       // single-tile kernel kept for comparison while the pipelined one is validated
-    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, out, ws, st) : launch_tc_attn<64>(g, tq, tk, tv, out, ws, st);
-  } else if (c->use_tc) {
+  if (c->use_tc && (cf.flags & 2u)) {       // previous kernel (no key split), kept for comparison while the new one is validated
     e = D == 128 ? launch_tc2_attn<128>(g, tq, tk, tv, out, ws, st) : launch_tc2_attn<64>(g, tq, tk, tv, out, ws, st);
+  } else if (c->use_tc) {
+    const int S = (cf.flags & 4u) ? 1 : attn_key_splits(g);
+    e = D == 128 ? launch_tc3_attn<128>(g, tq, tk, tv, out, ws, S, st) : launch_tc3_attn<64>(g, tq, tk, tv, out, ws, S, st);
   } else if (f32) {
     if (D == 128) launch_cc_attn<float, 128>(g, q, cache, out, ws, st); else launch_cc_attn<float, 64>(g, q, cache, out, ws, st);
   } else {

@@ -158,7 +158,11 @@ def test_layer_batched_call_matches_per_layer_calls():
                                out_b[:, pos0:pos0 + n])
     torch.cuda.synchronize()
     assert a.status() == 0 and b.status() == 0
-    assert torch.equal(out_a, out_b)
+    # the key range is split over more CTAs when fewer layers share a launch, so the two paths sum in a
+    # different order: outputs agree to bf16 rounding, not bit for bit
+    # (two bf16 roundings of nearly the same number may land one ulp apart: 2^-7 relative)
+    diff = (out_a.float() - out_b.float()).abs() / (out_a.float().abs() / 2).clamp_min(1.0)
+    assert diff.max().item() <= 2e-2
     for l in range(3):
         Ka, Va, Pa, la = a.cache_view(l); Kb, Vb, Pb, lb = b.cache_view(l)
         assert la == lb == cfg.budget

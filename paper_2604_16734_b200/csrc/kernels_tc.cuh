@@ -297,11 +297,14 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
 //   warps 0-3   softmax of tile A     (thread = one row = one TMEM lane), 216 registers
 //   warps 4-7   softmax of tile B
 //   warp  8     TMA producer: Q tiles once, then K_j, V_j, K_j+1, ... through a ring of kStages 32 KB slots
-//   warp  9     MMA issuer.  Per key tile j:  O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ; O_B += P_B V_j ;
-//               S_B = Q_B K_{j+1}^T, so the tensor pipe works on one row tile while the CUDA cores run
-//               the softmax of the other.  P is handed over in two halves (64 keys each) so the first
-//               PV MMAs start while the second half of the exponentials is still being computed.
-//   warps 10-11 only give their registers away (setmaxnreg works on groups of four warps)
+//   warp  9     MMA issuer of tile A, warp 10 of tile B (one lane each).  Per key tile j an issuer
+//               queues O_t += P_t V_j, then S_t = Q_t K_{j+1}^T.  P is handed over in two halves
+//               (64 keys each) so the first PV MMAs start while the second half of the exponentials
+//               is still being computed.
+//   warp  11    only gives its registers away (setmaxnreg works on groups of four warps)
+// The two softmax groups take turns (named barriers): while one tile's exponentials occupy the
+// CUDA cores the tensor pipe runs the other tile's MMAs; without the hand-over both tiles fall into
+// lockstep and the two pipes idle alternately.
 // TMEM columns: S_A/P_A [0,128)  S_B/P_B [128,256)  O_A [256,384)  O_B [384,512).
 // The running output is rescaled lazily: a row keeps its reference maximum until the true maximum
 // has grown by more than 2^8, so P stays below 256 and O rarely needs touching.
@@ -356,7 +359,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
       mbar_init(&sh.q_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.pv_done[i], 1);
       mbar_init(&sh.p_half[i][0], 128); mbar_init(&sh.p_half[i][1], 128);
     }
-    for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
+    // a ring slot is free again once the issuer of every active row tile has committed its MMAs on it
+    for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], has_B ? 2 : 1); }
     sh.abort_flag = 0;
     mbar_fence_init();
   }
@@ -406,65 +410,60 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
                         (t_begin + (i >> 1)) * 128, g, layer);
         }
       }
-    } else if (warp == 9) {
-      // ---------------------------------------------------------------- MMA issuer
+    } else if (warp == 9 || (warp == 10 && has_B)) {
+      // ---------------------------------------------------------------- MMA issuer of tile t
       if (lane == 0 && Tl > 0) {
-        const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
-        const uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
-        const uint32_t aQ = smem_u32(sQ), aR = smem_u32(ring);
-        auto issue_S = [&](int t, int slot) {      // S_t = Q_t K^T, 16 of the d columns per MMA
+        const int t = warp - 9;
+        constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
+        constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
+        constexpr uint32_t hi = smem_desc_hi_sw128(1024);
+        const uint32_t q_lo = smem_desc_lo(smem_u32(sQ) + t * TILE_BYTES, 16);          // K-major operand
+        const uint32_t k_lo0 = smem_desc_lo(smem_u32(ring), 16);                        // K-major operand
+        const uint32_t v_lo0 = smem_desc_lo(smem_u32(ring), kSubTileBytes);             // MN-major operand
+        const uint32_t tS = tmem + t * 128, tO = tmem + 256 + t * 128;
+        auto issue_S = [&](int slot) {             // S_t = Q_t K^T, 16 of the d columns per MMA
+          const uint32_t k_lo = k_lo0 + slot * (TILE_BYTES >> 4);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk / 4) * kSubTileBytes + (kk % 4) * 32;
-            mma_ss(tmem + t * 128, smem_desc_sw128(aQ + t * TILE_BYTES + off, 16, 1024),
-                   smem_desc_sw128(aR + slot * TILE_BYTES + off, 16, 1024), idesc_qk, kk > 0);
+            const uint32_t off = ((kk / 4) * kSubTileBytes + (kk % 4) * 32) >> 4;
+            mma_ss_lh(tS, q_lo + off, hi, k_lo + off, hi, idesc_qk, kk > 0);
           }
         };
-        auto issue_PV = [&](int t, int slot, int half, bool acc) {   // O_t += P_t V, 16 keys per MMA, 64 keys per half
+        auto issue_PV = [&](int slot, int half, bool acc) {   // O_t += P_t V, 16 keys per MMA, 64 keys per half
+          const uint32_t v_lo = v_lo0 + slot * (TILE_BYTES >> 4);
 #pragma unroll
           for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
-            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
-                   smem_desc_sw128(aR + slot * TILE_BYTES + kk * 2048, kSubTileBytes, 1024), idesc_pv, acc || kk > 0);
+            mma_ts_lh(tO, tS + kk * 8, v_lo + kk * (2048 >> 4), hi, idesc_pv, acc || kk > 0);
         };
-        bool ok = mbar_wait(&sh.q_full[0], 0, abort_flag) && mbar_wait(&sh.kv_full[0], 0, abort_flag);
+        bool ok = mbar_wait(&sh.q_full[t], 0, abort_flag) && mbar_wait(&sh.kv_full[0], 0, abort_flag);
         if (ok) {
           tc_fence_after_sync();
-          issue_S(0, 0);
-          mma_commit(&sh.s_full[0]);
-          if (has_B) {
-            ok = mbar_wait(&sh.q_full[1], 0, abort_flag);
-            if (ok) { issue_S(1, 0); mma_commit(&sh.s_full[1]); }
-          }
+          issue_S(0);
+          mma_commit(&sh.s_full[t]);
           mma_commit(&sh.kv_empty[0]);
         }
         for (int j = 0; j < Tl && ok; ++j) {
           const int iv = 2 * j + 1, ik = 2 * j + 2;
           const int slotV = iv % kStages, slotK = ik % kStages;
           const bool more = j + 1 < Tl;
-          for (int t = 0; t < (has_B ? 2 : 1) && ok; ++t) {
-            ok = mbar_wait(&sh.p_half[t][0], j & 1, abort_flag);
-            if (ok && t == 0) ok = mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after_sync();
-            issue_PV(t, slotV, 0, j > 0);
-            ok = mbar_wait(&sh.p_half[t][1], j & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after_sync();
-            issue_PV(t, slotV, 1, true);
-            mma_commit(&sh.pv_done[t]);
-            if (more) {
-              if (t == 0) {
-                ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after_sync();
-              }
-              issue_S(t, slotK);
-              mma_commit(&sh.s_full[t]);
-            }
-          }
+          ok = mbar_wait(&sh.p_half[t][0], j & 1, abort_flag) && mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
           if (!ok) break;
+          tc_fence_after_sync();
+          issue_PV(slotV, 0, j > 0);
+          ok = mbar_wait(&sh.p_half[t][1], j & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          issue_PV(slotV, 1, true);
+          mma_commit(&sh.pv_done[t]);
           mma_commit(&sh.kv_empty[slotV]);
-          if (more) mma_commit(&sh.kv_empty[slotK]);
+          if (more) {
+            ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            issue_S(slotK);
+            mma_commit(&sh.s_full[t]);
+            mma_commit(&sh.kv_empty[slotK]);
+          }
         }
       }
     }
@@ -484,11 +483,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const bool active = t == 0 || has_B;
+    // Turn taking (named barrier 2 + t = "tile t may go", 128 waiters + 128 arrivals).  Tile A goes first.
+    const bool turns = has_B && Tl > 0;
+    if (turns && t == 1) named_barrier_arrive(2, 256);
     if (active) {
       for (int j = 0; j < Tl; ++j) {
         const int kt = t_begin + j;                           // key tile index
-        ok = mbar_wait(&sh.s_full[t], j & 1, abort_flag);
-        if (!ok) break;
+        // Waits that gave up only skip the arithmetic: the turn barriers are passed on every path, once
+        // per key tile, so the other row tile never waits for a turn that is not handed over.
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[t], j & 1, abort_flag));
+        if (turns) named_barrier(2 + t, 256);
+        if (ok) do {
         tc_fence_after_sync();
         uint32_t sr[128];
 #pragma unroll
@@ -518,7 +523,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
           if (__any_sync(0xffffffffu, grow)) {
             const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;
             if (grow) { m_ref = m_new; l *= f; }
-            ok = mbar_wait(&sh.pv_done[t], (j - 1) & 1, abort_flag);   // O_t holds every earlier tile
+            ok = __all_sync(0xffffffffu, mbar_wait(&sh.pv_done[t], (j - 1) & 1, abort_flag));   // O_t holds every earlier tile
             if (!ok) break;
             tc_fence_after_sync();
 #pragma unroll
@@ -553,6 +558,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
           }
         }
         l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
+        } while (0);
+        if (turns && !(t == 1 && j + 1 == Tl)) named_barrier_arrive(3 - t, 256);
       }
       if (ok && Tl > 0) ok = mbar_wait(&sh.pv_done[t], (Tl - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);                       // the TMEM accesses below are warp-wide

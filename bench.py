@@ -35,7 +35,7 @@ from paper_2604_16734_b200.workloads import CONFIGS, Workload  # noqa: E402
 
 METRIC = "prefill tokens/s (attn+compress) per layer"
 UNIT = "tokens/s/layer"
-STEPS = ("append", "attention", "score", "select", "compact")
+STEPS = ("append", "attention", "score", "compress")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -54,7 +54,7 @@ def load_peaks():
 # ------------------------------------------------------------------------------------------------
 # algorithmic work of one launch (what the method itself has to move / compute)
 
-def work_of_call(cfg, n, n_c, moves_per_head=None):
+def work_of_call(cfg, n, n_c, moves_per_head=None, fused_score=True):
     """Bytes and FLOPs per step kind for ONE layer of one kvc_prefill_chunk call."""
     Hq, Hkv, d, sz, B = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.elem_bytes, cfg.budget
     tot = n_c + n
@@ -65,10 +65,15 @@ def work_of_call(cfg, n, n_c, moves_per_head=None):
                             flops=4 * Hq * d * (n * n_c + n * (n + 1) // 2))
     if tot > B:
         m = min(n, tot - B) * Hkv if moves_per_head is None else int(sum(moves_per_head))
-        out["score"] = dict(bytes=Hkv * (tot - w) * d * sz + Hq * w * d * sz + 4 * Hq * w + 4 * Hkv * (tot - w),
-                            flops=2 * Hq * w * d * (tot - w))
-        out["select"] = dict(bytes=2 * 4 * Hkv * (tot - w) + 8 * m, flops=0)
-        out["compact"] = dict(bytes=m * (2 * 2 * d * sz + 8 + 8), flops=0)
+        score = dict(bytes=Hkv * (tot - w) * d * sz + Hq * w * d * sz + 4 * Hq * w + 4 * Hkv * (tot - w),
+                     flops=2 * Hq * w * d * (tot - w))
+        select = 2 * 4 * Hkv * (tot - w) + 8 * m
+        compact = m * (2 * 2 * d * sz + 8 + 8)
+        if fused_score:          # one kernel scores, selects and compacts
+            out["compress"] = dict(bytes=score["bytes"] + select + compact, flops=score["flops"])
+        else:
+            out["score"] = score
+            out["compress"] = dict(bytes=select + compact, flops=0)
     return out
 
 
@@ -213,6 +218,7 @@ class Runner:
     def __init__(self, cfg, device_index, n_layers=None, flags=0):
         from paper_2604_16734_b200.binding import Kvc
         self.cfg = cfg
+        self.flags = flags
         self.L = cfg.n_layers if n_layers is None else n_layers
         self.dev = torch.device("cuda", device_index)
         wl = Workload(cfg, device=self.dev)
@@ -301,7 +307,8 @@ def profile_pass(r: Runner, steps: int):
             kv._check(kv._lib.kvc_prefill_chunk(kv._h, l, q, k, v, n, p, kv.cache[l].data_ptr(), kv.workspace.data_ptr(),
                                                 o, kv._stream()))
             moves = kv.move_counts(0).tolist() if n_c + n > cfg.budget else None
-            for s, wv in work_of_call(cfg, n, n_c, moves).items():
+            fused = cfg.dtype == "bf16" and not (r.flags & 1) and min(cfg.obs_window, n) * cfg.group <= 256
+            for s, wv in work_of_call(cfg, n, n_c, moves, fused).items():
                 work[s]["bytes"] += wv["bytes"]; work[s]["flops"] += wv["flops"]
         n_c = min(n_c + n, cfg.budget)
     torch.cuda.synchronize()

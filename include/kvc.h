@@ -190,8 +190,9 @@ int kvc_kv_bytes(const kvc_ctx* ctx, long long seq_len, size_t* logical, size_t*
 
 /* Per-kernel timing for measurement runs.  kvc_profile_enable(ctx, 1) makes every later call
  * bracket each of its kernels with a pair of CUDA events on the caller's stream (host objects, no
- * device memory).  kvc_profile_read synchronises those events and ADDS, per step index
- * (0 append, 1 attention, 2 score, 3 select, 4 compact), the elapsed milliseconds into ms[5] and
+ * device memory).  kvc_profile_read synchronises those events and ADDS, per kernel index
+ * (0 append, 1 attention, 2 score when it runs as a kernel of its own, 3 compress = select + compact,
+ * with the score inside when it is fused, 4 unused), the elapsed milliseconds into ms[5] and
  * the number of launches into launches[5] (both HOST arrays), then forgets the events.
  * Profiling perturbs end-to-end timing; leave it off in timed regions. */
 int kvc_profile_enable(kvc_ctx* ctx, int on);

@@ -261,7 +261,7 @@ class Kvc:
         ms = (ctypes.c_double * 5)()
         cnt = (ctypes.c_longlong * 5)()
         self._check(self._lib.kvc_profile_read(self._h, ms, cnt))
-        names = ("append", "attention", "score", "select", "compact")
+        names = ("append", "attention", "score", "compress", "unused")
         return dict(zip(names, list(ms))), dict(zip(names, list(cnt)))
 
     def launch_count(self) -> int:

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvc.so")
 SOURCES = ["kvc_api.cu"]
-HEADERS = ["geom.cuh", "ptx.cuh", "kernels_cc.cuh", "kernels_tc.cuh"]
+HEADERS = ["geom.cuh", "ptx.cuh", "kernels_cc.cuh", "kernels_tc.cuh", "compress.cuh"]
 
 
 def _stale() -> bool:

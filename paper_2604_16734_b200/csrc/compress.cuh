@@ -1,0 +1,389 @@
+// a2 + a3 + a4 in one launch: importance scores (Eq. 4), exact selection of the entries to evict
+// (Alg. 1, Evict) and hole-fill compaction back to the budget (Alg. 1, "reduce cache to budget M").
+//
+// One thread-block cluster of Cn CTAs per (kv-head, layer).
+//   phase 1 (SCORE = true, bf16)  the 128-key tiles of the candidates are dealt round-robin to the CTAs
+//            of the cluster.  Per tile: K tile by TMA, S^T = K_tile Q_obs^T on the tensor cores (keys on
+//            the TMEM lanes, observer rows on the columns), each thread sums 2^(s*scale - lse2) over
+//            the observer columns of its key and writes the score.  Two tiles are in flight per CTA
+//            (two K buffers, two TMEM accumulators, two epilogue warp groups).
+//            With SCORE = false the scores are already in the workspace (CUDA-core score kernel).
+//   phase 2  cluster barrier; then EVERY CTA reads all scores of its kv-head (L2-resident), builds the
+//            64-bit keys in shared memory and runs the same exact selection redundantly -- cheaper than
+//            a distributed histogram, since the SM-to-SM path is narrow and the other SMs would idle.
+//   phase 3  every CTA derives the same ordered hole / survivor lists and executes every Cn-th move.
+// Entry j gets the key (score bits << 32) | ~pos: a larger key means a higher score and, at equal
+// score, an older entry; keys are unique because positions are.  Scores are sums of probabilities,
+// hence >= 0, so their IEEE bit patterns order like integers.  The n_keep-th largest key (the cut-off)
+// is found exactly by an MSB-first radix descent with 12-bit digits that starts below the bits all
+// keys share and stops as soon as the bin that holds the cut-off survives as a whole.
+#pragma once
+#include <cuda.h>
+#include "geom.cuh"
+#include "ptx.cuh"
+
+namespace kvc {
+
+static constexpr int kCompressThreads = 1024;
+static constexpr int kSelBins = 4096;
+static constexpr int kMaxKeysSmem = 8192;     // candidates whose keys fit the shared-memory table (64 KB)
+static constexpr int kMaxMovesSmem = 4096;    // moves whose (src, dst) fit the shared-memory tables (32 KB)
+static constexpr int kSubTileBytesC = 128 * 128;
+
+__device__ __forceinline__ unsigned long long select_key(float score, int pos) {
+  return (static_cast<unsigned long long>(__float_as_uint(score)) << 32) |
+         static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(pos));
+}
+
+// The selection and the listing run on a team of kTeam threads (measured: a smaller team pays less per
+// barrier but more per key, and loses; the whole block it is).
+static constexpr int kTeam = kCompressThreads;
+__device__ __forceinline__ void team_sync() { named_barrier(3, kTeam); }
+
+// Inclusive scan of one int per team thread; returns the inclusive value and the team total.
+// scratch: kTeam / 32 + 1 ints of shared memory.  Only warp 0 combines the warp totals: a value that
+// every thread reads costs one load per warp, 32 of them cost 1024.
+__device__ __forceinline__ int team_scan_incl(int v, int* scratch, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  team_sync();                            // scratch may still be read from a previous scan
+  if (lane == 31) scratch[warp] = incl;
+  team_sync();
+  if (warp == 0) {
+    int t = scratch[lane], ti = t;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, ti, o);
+      if (lane >= o) ti += y;
+    }
+    scratch[lane] = ti - t;               // exclusive warp offsets
+    if (lane == 31) scratch[32] = ti;
+  }
+  team_sync();
+  *total = scratch[32];
+  return incl + scratch[warp];
+}
+
+struct CompressSmem {
+  uint64_t q_full, k_full[2], s_full[2], t_free[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  float lse2[256];
+  int hist[kSelBins];
+  unsigned long long list[2 * (kTeam / 32) + 2];
+  int scan_scratch[kTeam / 32 + 1];
+  unsigned long long s_prefix;
+  int s_remaining, s_bin_count;
+};
+
+// grid (Cn, Hkv, nl), cluster (Cn,1,1), block 1024.
+// dynamic smem: SCORE ? 2 * (D/64) * 16 KB + (D/64) * 32 KB + 1 KB : 96 KB + 1 KB (key and move tables).
+template <int D, bool SCORE>
+__global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __grid_constant__ CUtensorMap tm_k,
+                                                                       const __grid_constant__ CUtensorMap tm_qobs,
+                                                                       char* __restrict__ cache, char* __restrict__ ws,
+                                                                       Geom p, int Cn, int elem_bytes) {
+  constexpr int NSUB = D / 64;
+  constexpr int K_TILE_BYTES = NSUB * kSubTileBytesC;
+  constexpr int kQSubBytes = 256 * 128;          // up to 256 observer rows x 128 B
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ CompressSmem sh;
+
+  const int layer = blockIdx.z, g = blockIdx.y;
+  const int rank = Cn > 1 ? static_cast<int>(cluster_ctarank()) : 0;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  char* blob = cache + layer * p.cache_ls;
+  int* pos = reinterpret_cast<int*>(blob + p.pos_off) + static_cast<long long>(g) * p.cap;
+  char* slot = ws_slot(ws, p, layer);
+  float* score = reinterpret_cast<float*>(slot + p.score_off) + static_cast<long long>(g) * p.cap;
+  int* msrc_g = reinterpret_cast<int*>(slot + p.msrc_off) + static_cast<long long>(g) * p.max_chunk;
+  int* mdst_g = reinterpret_cast<int*>(slot + p.mdst_off) + static_cast<long long>(g) * p.max_chunk;
+  int* mcount = reinterpret_cast<int*>(slot + p.mcount_off);
+  volatile int* abort_flag = &sh.abort_flag;
+  if (tid == 0) sh.abort_flag = 0;
+
+  // ------------------------------------------------------------------------------------ phase 1: scores
+  if constexpr (SCORE) {
+    uint8_t* sK = smem;                              // two K tiles
+    uint8_t* sQ = smem + 2 * K_TILE_BYTES;           // observer rows
+    const int n_tiles = (p.n_cand + 127) / 128;
+    const int my_tiles = rank < n_tiles ? (n_tiles - rank + Cn - 1) / Cn : 0;
+    const int cols = p.w * p.G;                      // observer columns (<= 256: one MMA group)
+    const int n_mma = (cols + 15) & ~15;
+    if (tid == 0) {
+      mbar_init(&sh.q_full, 1);
+      for (int i = 0; i < 2; ++i) { mbar_init(&sh.k_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.t_free[i], 128); }
+      mbar_fence_init();
+    }
+    // observer rows beyond the real ones are padding: keep them finite
+    for (int i = tid; i < NSUB * kQSubBytes / 16; i += kCompressThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+    if (warp == 8) {
+      tmem_alloc(&sh.tmem_base, 512);
+      tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sh.tmem_base;
+    if (warp == 8) {
+      if (lane == 0) {
+        tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_qobs);
+        pdl_wait();
+        bool ok = true;
+        if (my_tiles > 0) {
+          mbar_expect_tx(&sh.q_full, NSUB * p.w * p.G * 128);
+          for (int sub = 0; sub < NSUB; ++sub)
+            tma_load_4d(sQ + sub * kQSubBytes, &tm_qobs, &sh.q_full, sub * 64, g * p.G, p.n - p.w, layer);
+          for (int i = 0; i < my_tiles && i < 2; ++i) {
+            mbar_expect_tx(&sh.k_full[i], K_TILE_BYTES);
+            for (int sub = 0; sub < NSUB; ++sub)
+              tma_load_4d(sK + i * K_TILE_BYTES + sub * kSubTileBytesC, &tm_k, &sh.k_full[i], sub * 64,
+                          (rank + i * Cn) * 128, g, layer);
+          }
+          ok = mbar_wait(&sh.q_full, 0, abort_flag);
+        }
+        const uint32_t idesc = idesc_bf16_f32(128, n_mma, 0, 0);
+        constexpr uint32_t hi = smem_desc_hi_sw128(1024);
+        const uint32_t k_lo0 = smem_desc_lo(smem_u32(sK), 16), q_lo = smem_desc_lo(smem_u32(sQ), 16);
+        for (int i = 0; i < my_tiles && ok; ++i) {
+          const int b = i & 1;
+          ok = mbar_wait(&sh.k_full[b], (i >> 1) & 1, abort_flag);
+          if (ok && i >= 2) ok = mbar_wait(&sh.t_free[b], ((i - 2) >> 1) & 1, abort_flag);   // accumulator b read out
+          if (!ok) break;
+          tc_fence_after_sync();
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss_lh(tmem + b * 256, k_lo0 + ((b * K_TILE_BYTES + (kk / 4) * kSubTileBytesC + (kk % 4) * 32) >> 4), hi,
+                      q_lo + (((kk / 4) * kQSubBytes + (kk % 4) * 32) >> 4), hi, idesc, kk > 0);
+          mma_commit(&sh.s_full[b]);
+          if (i + 2 < my_tiles) {                    // refill K buffer b once the MMAs that read it are done
+            ok = mbar_wait(&sh.s_full[b], (i >> 1) & 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(&sh.k_full[b], K_TILE_BYTES);
+            for (int sub = 0; sub < NSUB; ++sub)
+              tma_load_4d(sK + b * K_TILE_BYTES + sub * kSubTileBytesC, &tm_k, &sh.k_full[b], sub * 64,
+                          (rank + (i + 2) * Cn) * 128, g, layer);
+          }
+        }
+      }
+      __syncwarp();
+    } else if (warp < 8) {
+      const int b = warp >> 2;
+      const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+      pdl_wait();
+      const float* lse = reinterpret_cast<const float*>(slot + p.lse_off);
+      // log-sum-exp of the observer rows in log2 units; padding columns get +inf (2^-inf = 0).
+      // Each epilogue group fills the whole table (same values), so no cross-group barrier is needed.
+      for (int c = (warp & 3) * 32 + lane; c < 256; c += 128) {
+        float lv = INFINITY;
+        if (c < cols) lv = lse[static_cast<long long>(p.n - p.w + c / p.G) * p.Hq + g * p.G + c % p.G] * 1.4426950408889634f;
+        sh.lse2[c] = lv;
+      }
+      named_barrier(1 + b, 128);
+      bool ok = true;
+      for (int i = b; i < my_tiles; i += 2) {
+        ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[b], (i >> 1) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after_sync();
+        float acc = 0.f;
+        float acc2 = 0.f;
+        for (int c0 = 0; c0 < n_mma; c0 += 32) {       // n_mma is a multiple of 16: the second half may be absent
+          uint32_t sr[32];
+          const bool two = c0 + 16 < n_mma;
+          tmem_ld16(tmem + b * 256 + lane_addr + c0, sr);
+          if (two) tmem_ld16(tmem + b * 256 + lane_addr + c0 + 16, sr + 16);
+          tmem_wait_ld();
+#pragma unroll
+          for (int k = 0; k < 16; ++k) acc += fast_exp2(fmaf(__uint_as_float(sr[k]), p.scale_log2, -sh.lse2[c0 + k]));
+          if (two) {
+#pragma unroll
+            for (int k = 16; k < 32; ++k) acc2 += fast_exp2(fmaf(__uint_as_float(sr[k]), p.scale_log2, -sh.lse2[c0 + k]));
+          }
+        }
+        acc += acc2;
+        tc_fence_before_sync();
+        mbar_arrive(&sh.t_free[b]);
+        const int key = (rank + i * Cn) * 128 + (warp & 3) * 32 + lane;
+        if (key < p.n_cand) score[key] = acc;
+      }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 8) {
+      tc_fence_after_sync();
+      tmem_dealloc(tmem, 512);
+    }
+  } else {
+    if (tid == 0) pdl_wait();
+    __syncthreads();
+  }
+  if (Cn > 1) {                                       // every score of this kv-head is in the workspace
+    cluster_arrive();
+    cluster_wait();
+  } else {
+    __syncthreads();
+  }
+
+  // ------------------------------------------------------------------------------------ phase 2: selection
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);           // 64 KB
+  int* tab_src = reinterpret_cast<int*>(smem + kMaxKeysSmem * 8);                    // 16 KB
+  int* tab_dst = tab_src + kMaxMovesSmem;                                            // 16 KB
+  const bool keys_in_smem = p.n_cand <= kMaxKeysSmem;
+  if (keys_in_smem)
+    for (int j = tid; j < p.n_cand; j += kCompressThreads) keys[j] = select_key(__ldcg(score + j), pos[j]);
+  __syncthreads();
+  auto key_of = [&](int j) -> unsigned long long {
+    return keys_in_smem ? keys[j] : select_key(__ldcg(score + j), pos[j]);
+  };
+
+  if (p.n_keep > 0) {
+    {                                                            // (all kTeam threads)
+      // The bits above the highest bit in which any two keys differ are common to all keys (scores of
+      // similar magnitude share their exponent bits): start the descent below them, so that the first
+      // digit already spreads the keys over many bins instead of piling them onto a few counters.
+      unsigned long long k_and = ~0ull, k_or = 0ull;
+      for (int j = tid; j < p.n_cand; j += kTeam) { const unsigned long long k = key_of(j); k_and &= k; k_or |= k; }
+      unsigned a_lo = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(k_and)), a_hi = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(k_and >> 32));
+      unsigned o_lo = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or)), o_hi = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or >> 32));
+      if (lane == 0) { sh.list[warp] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[kTeam / 32 + warp] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
+      team_sync();
+      if (warp == 0) {                                           // one warp folds the 32 partial results
+        const unsigned long long pa = sh.list[lane], po = sh.list[kTeam / 32 + lane];
+        a_lo = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(pa)); a_hi = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(pa >> 32));
+        o_lo = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(po)); o_hi = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(po >> 32));
+        if (lane == 0) { sh.list[2 * (kTeam / 32)] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[2 * (kTeam / 32) + 1] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
+      }
+      team_sync();
+      k_and = sh.list[2 * (kTeam / 32)]; k_or = sh.list[2 * (kTeam / 32) + 1];
+      const unsigned long long differ = k_and ^ k_or;           // != 0: at least two distinct keys (n_cand > n_keep >= 1)
+      const int top = 63 - __clzll(static_cast<long long>(differ));
+      int shift = top >= 11 ? top - 11 : 0, bits = top - shift + 1;
+      team_sync();                                               // sh.list is reused below
+      if (tid == 0) { sh.s_prefix = top == 63 ? 0ull : (k_or >> (top + 1)) << (top + 1); sh.s_remaining = p.n_keep; }
+      while (true) {
+        for (int i = tid; i < kSelBins; i += kTeam) sh.hist[i] = 0;
+        team_sync();
+        const unsigned long long prefix = sh.s_prefix;
+        const int remaining = sh.s_remaining;
+        const int hi = shift + bits;         // bits [hi, 64) are already decided
+        for (int j = tid; j < p.n_cand; j += kTeam) {
+          const unsigned long long key = key_of(j);
+          if (hi >= 64 || (key >> hi) == (prefix >> hi)) atomicAdd(&sh.hist[(key >> shift) & ((1u << bits) - 1)], 1);
+        }
+        team_sync();
+        // descending scan: thread t owns the BPT bins from 4095 - BPT*t downwards
+        constexpr int BPT = kSelBins / kTeam;
+        const int b0 = kSelBins - 1 - BPT * tid;
+        int mine = 0;
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) mine += sh.hist[b0 - i];
+        int total;
+        const int incl = team_scan_incl(mine, sh.scan_scratch, &total);
+        int excl = incl - mine;
+        if (excl < remaining && remaining <= incl) {             // the cut-off lies in one of my bins
+          int b = b0, h = sh.hist[b0];
+          while (excl + h < remaining) { excl += h; --b; h = sh.hist[b]; }
+          sh.s_prefix = prefix | (static_cast<unsigned long long>(b) << shift);
+          sh.s_remaining = remaining - excl;                     // rank inside the chosen bin, 1-based
+          sh.s_bin_count = h;
+        }
+        team_sync();
+        // Done when every bit is decided, or when the whole bin survives (its rank equals its size): then
+        // the prefix with zeros below it separates the retained keys from the others.
+        if (shift == 0 || sh.s_remaining == sh.s_bin_count) break;
+        bits = shift >= 12 ? 12 : shift;
+        shift -= bits;
+      }
+    }
+    __syncthreads();
+  }
+  const unsigned long long thr = p.n_keep > 0 ? sh.s_prefix : ~0ull;   // n_keep == 0: nothing among the candidates survives
+
+  // ------------------------------------------------------------------------------------ phase 3: compaction
+  // holes: evicted entries in rows [0, B); survivors: retained entries in rows [B, tot), both in ascending
+  // row order.  Entry j is retained iff it is protected (j >= n_cand) or its key >= thr.
+  const int n_lo = min(p.B, p.tot);
+  const int max_moves = min(p.n, p.tot - p.B);                   // at most this many entries sit at or above row B
+  const bool tabs_in_smem = max_moves <= kMaxMovesSmem;
+  int* msrc = tabs_in_smem ? tab_src : msrc_g;                   // with global tables every CTA writes all entries
+  int* mdst = tabs_in_smem ? tab_dst : mdst_g;                   // itself (same values) and reads only its own writes
+  {
+    // Each warp owns a contiguous segment of the rows, walked 32 rows at a time (lane = row, so the
+    // shared-memory keys are read without bank conflicts).  Pass 1 counts the warp's holes (rows below
+    // B) and survivors (rows from B on), one scan over the 32 warps turns the counts into offsets,
+    // pass 2 writes the row indices in ascending order.
+    const int seg = ((p.tot + 31) / 32 + 31) & ~31;              // rows per warp, a multiple of 32
+    const int s0 = warp * seg, s1 = min(s0 + seg, p.tot);
+    auto retained = [&](int j) { return j >= p.n_cand || key_of(j) >= thr; };
+    int holes = 0, surv = 0;
+    for (int base = s0; base < s1; base += 32) {
+      const int j = base + lane;
+      const bool valid = j < s1;
+      const bool keep = valid && retained(j);
+      holes += __popc(__ballot_sync(0xffffffffu, valid && j < n_lo && !keep));
+      surv += __popc(__ballot_sync(0xffffffffu, valid && j >= n_lo && keep));
+    }
+    // both counts share one scan when they fit 16 bits each (tot < 65536); lane 0 carries the warp's counts
+    int total_holes, off_h, off_s;
+    if (p.tot < 65536) {
+      int total;
+      const int mine = lane == 0 ? (holes | (surv << 16)) : 0;
+      const int packed = team_scan_incl(mine, sh.scan_scratch, &total);
+      off_h = __shfl_sync(0xffffffffu, (packed & 0xffff) - holes, 0);
+      off_s = __shfl_sync(0xffffffffu, (packed >> 16) - surv, 0);
+      total_holes = total & 0xffff;
+    } else {
+      int total_surv;
+      off_h = __shfl_sync(0xffffffffu, team_scan_incl(lane == 0 ? holes : 0, sh.scan_scratch, &total_holes) - holes, 0);
+      off_s = __shfl_sync(0xffffffffu, team_scan_incl(lane == 0 ? surv : 0, sh.scan_scratch, &total_surv) - surv, 0);
+    }
+    for (int base = s0; base < s1; base += 32) {
+      const int j = base + lane;
+      const bool valid = j < s1;
+      const bool keep = valid && retained(j);
+      const bool is_hole = valid && j < n_lo && !keep, is_surv = valid && j >= n_lo && keep;
+      const unsigned mh = __ballot_sync(0xffffffffu, is_hole), ms = __ballot_sync(0xffffffffu, is_surv);
+      const unsigned below = (1u << lane) - 1;
+      if (is_hole) mdst[off_h + __popc(mh & below)] = j;
+      if (is_surv) msrc[off_s + __popc(ms & below)] = j;
+      off_h += __popc(mh);
+      off_s += __popc(ms);
+    }
+    if (tid == 0) sh.s_remaining = total_holes;                  // == number of survivors: the cache returns to B
+  }
+  __syncthreads();
+  const int total_holes = sh.s_remaining;
+  if (rank == 0 && tid == 0) mcount[g] = total_holes;
+  if (Cn > 1) {                                                  // the moves overwrite positions (and rows) that the
+    cluster_arrive();                                            // other CTAs of the cluster read while selecting
+    cluster_wait();
+  }
+
+  // move m copies the K row, the V row and the position of entry src[m] (>= B) into the hole dst[m] (< B).
+  // Sources and destinations never overlap, rows are copied bit-exactly.  One warp per move.
+  const long long row_bytes = static_cast<long long>(p.d) * elem_bytes;
+  const int vec = static_cast<int>(row_bytes / 16);
+  const long long head = static_cast<long long>(g) * p.cap;
+  for (int mv = rank * (kCompressThreads / 32) + warp; mv < total_holes; mv += Cn * (kCompressThreads / 32)) {
+    const int src = msrc[mv], dst = mdst[mv];
+    const uint4* ks = reinterpret_cast<const uint4*>(blob + (head + src) * row_bytes);
+    const uint4* vs = reinterpret_cast<const uint4*>(blob + p.v_off + (head + src) * row_bytes);
+    uint4* kd = reinterpret_cast<uint4*>(blob + (head + dst) * row_bytes);
+    uint4* vd = reinterpret_cast<uint4*>(blob + p.v_off + (head + dst) * row_bytes);
+    for (int i = lane; i < 2 * vec; i += 32) {
+      if (i < vec) kd[i] = ks[i];
+      else vd[i - vec] = vs[i - vec];
+    }
+    if (lane == 0) pos[dst] = pos[src];
+  }
+  if (tid == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+}
+
+}  // namespace kvc

@@ -1,5 +1,5 @@
 // CUDA-core kernels: append (a0), fp32-accurate attention (a1) and score (a2) for fp32 inputs
-// (and, as a diagnostic, bf16 inputs), exact per-head selection (a3) and hole-fill compaction (a4).
+// (and, as a diagnostic, bf16 inputs).
 #pragma once
 #include "geom.cuh"
 
@@ -210,174 +210,6 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
   }
   const int key = key0 + threadIdx.x;
   if (key < p.n_cand) score[key] = acc;
-}
-
-// ------------------------------------------------------------------------------------------------
-// a3 select (Alg. 1 Evict): one CTA per (kv-head, layer).  Entry j gets the 64-bit key
-// (score bits << 32) | ~pos, so a larger key means a higher score and, at equal score, an older
-// entry; keys are unique because positions are.  Scores are sums of probabilities, hence >= 0, so
-// their IEEE bit patterns order like integers.  The n_keep-th largest key (the cut-off) is found
-// exactly by an MSB-first radix descent with 12-bit digits; as soon as the bin that holds the
-// cut-off has at most kListCap members they are gathered into shared memory and ranked by direct
-// comparison.  Two block scans then produce, in ascending row order, the holes (evicted rows below
-// B) and the survivors (retained rows at or above B) that compaction pairs up.
-// grid (Hkv, 1, nl), block 1024.
-__device__ __forceinline__ unsigned long long select_key(float score, int pos) {
-  return (static_cast<unsigned long long>(__float_as_uint(score)) << 32) |
-         static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(pos));
-}
-
-static constexpr int kSelBins = 4096;
-static constexpr int kListCap = 512;
-
-// Inclusive scan of one int per thread over a 1024-thread block; returns the inclusive value and
-// the block total.  scratch: 33 ints of shared memory.
-__device__ __forceinline__ int block_scan_incl(int v, int* scratch, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
-  }
-  __syncthreads();                        // scratch may still be read from a previous scan
-  if (lane == 31) scratch[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    int t = scratch[lane], ti = t;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, ti, o);
-      if (lane >= o) ti += y;
-    }
-    scratch[lane] = ti - t;               // exclusive warp offsets
-    if (lane == 31) scratch[32] = ti;
-  }
-  __syncthreads();
-  *total = scratch[32];
-  return incl + scratch[warp];
-}
-
-__global__ void __launch_bounds__(1024) select_kernel(const char* __restrict__ cache, char* __restrict__ ws, Geom p) {
-  __shared__ int hist[kSelBins];
-  __shared__ unsigned long long list[kListCap];
-  __shared__ int scan_scratch[33];
-  __shared__ unsigned long long s_prefix;
-  __shared__ int s_remaining, s_bin_count, s_nlist;
-  const int layer = blockIdx.z, g = blockIdx.x;
-  const int tid = threadIdx.x;
-  const char* blob = cache + layer * p.cache_ls;
-  const int* pos = reinterpret_cast<const int*>(blob + p.pos_off) + static_cast<long long>(g) * p.cap;
-  char* slot = ws_slot(ws, p, layer);
-  const float* score = reinterpret_cast<const float*>(slot + p.score_off) + static_cast<long long>(g) * p.cap;
-  int* msrc = reinterpret_cast<int*>(slot + p.msrc_off) + static_cast<long long>(g) * p.max_chunk;
-  int* mdst = reinterpret_cast<int*>(slot + p.mdst_off) + static_cast<long long>(g) * p.max_chunk;
-  int* mcount = reinterpret_cast<int*>(slot + p.mcount_off);
-
-  unsigned long long thr = ~0ull;            // n_keep == 0: nothing among the candidates survives
-  if (p.n_keep > 0) {
-    if (tid == 0) { s_prefix = 0ull; s_remaining = p.n_keep; s_nlist = 0; }
-    int shift = 52, bits = 12;
-    while (true) {
-      for (int i = tid; i < kSelBins; i += 1024) hist[i] = 0;
-      __syncthreads();
-      const unsigned long long prefix = s_prefix;
-      const int remaining = s_remaining;
-      const int hi = shift + bits;           // bits [hi, 64) are already decided
-      for (int j = tid; j < p.n_cand; j += 1024) {
-        const unsigned long long key = select_key(score[j], pos[j]);
-        if (hi >= 64 || (key >> hi) == (prefix >> hi)) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1)], 1);
-      }
-      __syncthreads();
-      // descending scan: thread t owns bins 4095-4t .. 4092-4t
-      const int b0 = kSelBins - 1 - 4 * tid;
-      const int h0 = hist[b0], h1 = hist[b0 - 1], h2 = hist[b0 - 2], h3 = hist[b0 - 3];
-      int total;
-      const int incl = block_scan_incl(h0 + h1 + h2 + h3, scan_scratch, &total);
-      int excl = incl - (h0 + h1 + h2 + h3);
-      if (excl < remaining && remaining <= incl) {               // the cut-off lies in one of my four bins
-        int b = b0, h = h0;
-        if (excl + h < remaining) { excl += h; b = b0 - 1; h = h1;
-          if (excl + h < remaining) { excl += h; b = b0 - 2; h = h2;
-            if (excl + h < remaining) { excl += h; b = b0 - 3; h = h3; } } }
-        s_prefix = prefix | (static_cast<unsigned long long>(b) << shift);
-        s_remaining = remaining - excl;                          // rank inside the chosen bin, 1-based
-        s_bin_count = h;
-      }
-      __syncthreads();
-      if (shift == 0) { thr = s_prefix; break; }                 // every bit decided
-      if (s_bin_count <= kListCap) {
-        // gather the bin's members and rank them directly
-        const unsigned long long pre = s_prefix;
-        for (int j = tid; j < p.n_cand; j += 1024) {
-          const unsigned long long key = select_key(score[j], pos[j]);
-          if ((key >> shift) == (pre >> shift)) list[atomicAdd(&s_nlist, 1)] = key;
-        }
-        __syncthreads();
-        const int m = s_nlist, want = s_remaining - 1;
-        if (tid < m) {
-          const unsigned long long mine = list[tid];
-          int greater = 0;
-          for (int f = 0; f < m; ++f) greater += list[f] > mine;
-          if (greater == want) s_prefix = mine;                  // exactly one element has this rank
-        }
-        __syncthreads();
-        thr = s_prefix;
-        break;
-      }
-      bits = shift >= 12 ? 12 : shift;
-      shift -= bits;
-    }
-  }
-
-  // ---- holes: evicted entries in rows [0, B); survivors: retained entries in rows [B, tot).
-  // Entry j is retained iff it is protected (j >= n_cand) or its key >= thr.
-  const int n_lo = min(p.B, p.tot), n_hi = p.tot - n_lo;
-  const int per_lo = (n_lo + 1023) / 1024, per_hi = (n_hi + 1023) / 1024;
-  const int a0 = min(tid * per_lo, n_lo), a1 = min(a0 + per_lo, n_lo);
-  const int c0 = n_lo + min(tid * per_hi, n_hi), c1 = min(c0 + per_hi, p.tot);
-  int holes = 0, surv = 0;
-  for (int j = a0; j < a1; ++j) holes += !(j >= p.n_cand || select_key(score[j], pos[j]) >= thr);
-  for (int j = c0; j < c1; ++j) surv += (j >= p.n_cand || select_key(score[j], pos[j]) >= thr);
-  int total_holes, total_surv;
-  int rank_h = block_scan_incl(holes, scan_scratch, &total_holes) - holes;
-  int rank_s = block_scan_incl(surv, scan_scratch, &total_surv) - surv;
-  for (int j = a0; j < a1; ++j)
-    if (!(j >= p.n_cand || select_key(score[j], pos[j]) >= thr)) mdst[rank_h++] = j;
-  for (int j = c0; j < c1; ++j)
-    if (j >= p.n_cand || select_key(score[j], pos[j]) >= thr) msrc[rank_s++] = j;
-  if (tid == 0) mcount[g] = total_holes;                         // == total_surv: the cache returns to B
-}
-
-// ------------------------------------------------------------------------------------------------
-// a4 compact: move m copies the K row, the V row and the position of entry src[m] (>= B) into the
-// hole dst[m] (< B).  Sources and destinations never overlap, rows are copied bit-exactly.
-// One warp per move.  grid (ceil(max_moves/8), Hkv, nl), block 256.
-__global__ void __launch_bounds__(256) compact_kernel(char* __restrict__ cache, const char* __restrict__ ws, Geom p,
-                                                      int elem_bytes) {
-  const int layer = blockIdx.z, g = blockIdx.y;
-  const int mv = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  const char* slot = ws + kWsHeaderBytes + static_cast<long long>(layer) * p.ws_ls;
-  const int count = reinterpret_cast<const int*>(slot + p.mcount_off)[g];
-  if (mv >= count) return;
-  const int src = reinterpret_cast<const int*>(slot + p.msrc_off)[static_cast<long long>(g) * p.max_chunk + mv];
-  const int dst = reinterpret_cast<const int*>(slot + p.mdst_off)[static_cast<long long>(g) * p.max_chunk + mv];
-  char* blob = cache + layer * p.cache_ls;
-  const long long row_bytes = static_cast<long long>(p.d) * elem_bytes;
-  const int vec = static_cast<int>(row_bytes / 16);
-  const long long head = static_cast<long long>(g) * p.cap;
-  const uint4* ks = reinterpret_cast<const uint4*>(blob + (head + src) * row_bytes);
-  const uint4* vs = reinterpret_cast<const uint4*>(blob + p.v_off + (head + src) * row_bytes);
-  uint4* kd = reinterpret_cast<uint4*>(blob + (head + dst) * row_bytes);
-  uint4* vd = reinterpret_cast<uint4*>(blob + p.v_off + (head + dst) * row_bytes);
-  for (int i = lane; i < 2 * vec; i += 32) {
-    if (i < vec) kd[i] = ks[i];
-    else vd[i - vec] = vs[i - vec];
-  }
-  if (lane == 0) {
-    int* pp = reinterpret_cast<int*>(blob + p.pos_off) + head;
-    pp[dst] = pp[src];
-  }
 }
 
 }  // namespace kvc

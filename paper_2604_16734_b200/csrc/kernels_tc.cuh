@@ -311,9 +311,9 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
 //
 // Key split: with cluster size S the CTA of cluster rank s handles key tiles [s*T/S, (s+1)*T/S) of
 // its row-tile pair and ends with a partial (O, m, l).  The partials are exchanged through
-// distributed shared memory: every CTA parks its O tiles (fp32, column-major so that lanes write
-// consecutive words) in its own ring buffer, the cluster synchronises, and rank s combines and
-// writes rows [s*128/S, (s+1)*128/S) of both tiles.  Nothing but the final result goes to HBM.
+// distributed shared memory: rank s owns rows [s*128/S, (s+1)*128/S) of both tiles, every CTA pushes
+// its partial rows (fp32) into the owner's shared memory with remote stores, the cluster
+// synchronises, and each rank combines and writes its rows.  Nothing but the final result goes to HBM.
 // grid (ceil(ceil(n/TOK)/2) * S, Hkv, nl), cluster (S,1,1), block 384,
 // dynamic smem (2 + kStages) * (D/64) * 16 KB + 1 KB.
 static constexpr int kAttnThreads = 384;
@@ -322,7 +322,6 @@ struct TcSmemAttn3 {
   uint64_t q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_half[2][2], pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
-  float stat_m[2][128], stat_l[2][128];   // per row: reference maximum (log2 units, -inf if the row saw no key) and sum
 };
 
 template <int D>
@@ -468,6 +467,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
       }
     }
     __syncwarp();
+    if (S > 1) {                                             // the two cluster barriers of the combine below
+      cluster_arrive(); cluster_wait();
+      cluster_arrive(); cluster_wait();
+    }
   } else {
     reg_inc<216>();
     // ---------------------------------------------------------------- softmax + epilogue of tile t
@@ -480,7 +483,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
     const int tile_min_limit = p.n_c + tok0 + 1;              // smallest limit of any row of the tile
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tmem_S = tmem + t * 128 + lane_addr, tmem_O = tmem + 256 + t * 128 + lane_addr;
-    float m_ref = -INFINITY, l = 0.f;
+    float m_ref = -INFINITY, l = 0.f;                        // reference maximum (log2 units) and row sum
     bool ok = true;
     const bool active = t == 0 || has_B;
     // Turn taking (named barrier 2 + t = "tile t may go", 128 waiters + 128 arrivals).  Tile A goes first.
@@ -590,89 +593,109 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
             lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_ref + log2f(l)) * 0.6931471805599453f;
           }
         }
-      } else {
-        // park this CTA's partial of tile t: O column-major [D][128] fp32 in the ring, m and l beside the barriers.
-        // Every MMA of the CTA (both tiles) has to be complete before the ring is overwritten.
-        if (has_B) named_barrier(1, 256);
-        float* stg = reinterpret_cast<float*>(ring) + t * (D * 128);
-        if (ok && Tl > 0) {
+      }
+    }
+    if (S > 1) {
+      // Combine the partials of the cluster.  Rank s owns rows [s*rows_per, (s+1)*rows_per) of both tiles.
+      // Every softmax thread pushes its row of O (fp32: the output tolerance leaves no room for a 16-bit
+      // exchange format) and its (m, l) into the owner's shared memory with remote stores -- stores are
+      // not waited for, remote loads would be; rows it owns itself are stored locally -- the cluster
+      // synchronises, and each rank reduces its rows from its own shared memory:
+      //   O = sum_s 2^(m_s - m*) O_s / sum_s 2^(m_s - m*) l_s.
+      // stage: [S sources][2 tiles][rows_per][D] fp32 over the Q tiles and the ring; the 16-byte chunks of
+      // a row are XOR-swizzled with (row & 7) so that neither the writers (lane = row) nor the readers
+      // (lane = row, same chunk) collide on banks.
+      const int rows_per = (128 + S - 1) / S;
+      float* stage = reinterpret_cast<float*>(smem);
+      float* stat = stage + S * 2 * rows_per * D;               // [S][2][rows_per][2]: m (-inf: row saw no key), l
+      cluster_arrive();                                         // every CTA is done with its Q tiles and ring
+      cluster_wait();
+      if (active) {
+        const int owner = r / rows_per, lr = r - owner * rows_per;
+        const int slot = ((split * 2 + t) * rows_per + lr);
+        uint32_t row_addr = smem_u32(stage + slot * D), stat_addr = smem_u32(stat + slot * 2);
+        if (owner != split) { row_addr = dsmem_addr(row_addr, owner); stat_addr = dsmem_addr(stat_addr, owner); }
+        const bool have = ok && Tl > 0;                         // warp-uniform
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          if (have) {
             tmem_ld32(tmem_O + c * 32, o);
             tmem_wait_ld();
+          } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) stg[(c * 32 + i) * 128 + r] = __uint_as_float(o[i]);
+            for (int i = 0; i < 32; ++i) o[i] = 0u;
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            dsmem_st_v4_b32(row_addr + (((c * 8 + k) ^ (lr & 7)) << 4), o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+        }
+        dsmem_st_v2(stat_addr, (have && l > 0.f) ? m_ref : -INFINITY, have ? l : 0.f);
+      }
+      cluster_arrive();                                         // all partials have landed; no remote access after this
+      cluster_wait();
+      {
+        const int r0 = min(128, split * rows_per), nrows = min(128, r0 + rows_per) - r0;
+        const int per_tile = nrows * (D / 32);                  // work items: (row, group of 32 columns)
+        for (int item = threadIdx.x; item < (has_B ? 2 : 1) * per_tile; item += 256) {
+          const int t = item / per_tile, rem = item % per_tile;
+          const int lr = rem % nrows, cg = rem / nrows, r = r0 + lr;
+          const int tok = (t ? tokB : tokA) + r / p.G, hh = r % p.G;
+          if (!(r < rows && tok < p.n)) continue;
+          float ms[8], wt[8];
+          float m_all = -INFINITY;
+#pragma unroll
+          for (int s = 0; s < 8; ++s) {
+            ms[s] = -INFINITY;
+            if (s < S) ms[s] = stat[((s * 2 + t) * rows_per + lr) * 2];
+            m_all = fmaxf(m_all, ms[s]);
+          }
+          float L = 0.f;
+#pragma unroll
+          for (int s = 0; s < 8; ++s) {
+            wt[s] = 0.f;
+            if (s < S && ms[s] != -INFINITY) {
+              wt[s] = fast_exp2(ms[s] - m_all);
+              L = fmaf(wt[s], stat[((s * 2 + t) * rows_per + lr) * 2 + 1], L);
+            }
+          }
+          float acc[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll
+          for (int s = 0; s < 8; ++s) {
+            if (s < S && wt[s] != 0.f) {
+              const float* row = stage + ((s * 2 + t) * rows_per + lr) * D;
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const float4 v4 = *reinterpret_cast<const float4*>(row + (((cg * 8 + k) ^ (lr & 7)) << 2));
+                acc[4 * k + 0] = fmaf(wt[s], v4.x, acc[4 * k + 0]);
+                acc[4 * k + 1] = fmaf(wt[s], v4.y, acc[4 * k + 1]);
+                acc[4 * k + 2] = fmaf(wt[s], v4.z, acc[4 * k + 2]);
+                acc[4 * k + 3] = fmaf(wt[s], v4.w, acc[4 * k + 3]);
+              }
+            }
+          }
+          const float inv = 1.f / L;
+          __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D + cg * 32;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 vv;
+            vv.x = pack_bf16x2(acc[8 * i + 0] * inv, acc[8 * i + 1] * inv);
+            vv.y = pack_bf16x2(acc[8 * i + 2] * inv, acc[8 * i + 3] * inv);
+            vv.z = pack_bf16x2(acc[8 * i + 4] * inv, acc[8 * i + 5] * inv);
+            vv.w = pack_bf16x2(acc[8 * i + 6] * inv, acc[8 * i + 7] * inv);
+            reinterpret_cast<uint4*>(orow)[i] = vv;
+          }
+          if (cg == 0) {
+            float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
+            lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_all + log2f(L)) * 0.6931471805599453f;
           }
         }
-        sh.stat_m[t][r] = (ok && l > 0.f) ? m_ref : -INFINITY;
-        sh.stat_l[t][r] = l;
       }
     }
   }
 
-  if (S > 1) {
-    cluster_arrive();                                         // partials of every rank are in place
-    cluster_wait();
-    if (warp < 8) {
-      // rank `split` combines rows [r0, r1) of both tiles: O = sum_s 2^(m_s - m*) O_s / sum_s 2^(m_s - m*) l_s
-      const int rows_per = (128 + S - 1) / S;
-      const int r0 = min(128, split * rows_per), r1 = min(128, r0 + rows_per), nrows = r1 - r0;
-      const int per_tile = nrows * (D / 32);                  // work items: (row, group of 32 columns)
-      const uint32_t a_stg = smem_u32(ring), a_m = smem_u32(&sh.stat_m[0][0]), a_l = smem_u32(&sh.stat_l[0][0]);
-      for (int item = threadIdx.x; item < (has_B ? 2 : 1) * per_tile; item += 256) {
-        const int t = item / per_tile, rem = item % per_tile;
-        const int r = r0 + rem % nrows, cg = rem / nrows;
-        const int tok = (t ? tokB : tokA) + r / p.G, hh = r % p.G;
-        if (!(r < rows && tok < p.n)) continue;
-        float ms[8], wt[8];
-        float m_all = -INFINITY;
-#pragma unroll
-        for (int s = 0; s < 8; ++s) {
-          ms[s] = -INFINITY;
-          if (s < S) ms[s] = dsmem_ld_f32(dsmem_addr(a_m + (t * 128 + r) * 4, s));
-          m_all = fmaxf(m_all, ms[s]);
-        }
-        float L = 0.f;
-#pragma unroll
-        for (int s = 0; s < 8; ++s) {
-          wt[s] = 0.f;
-          if (s < S && ms[s] != -INFINITY) {
-            wt[s] = fast_exp2(ms[s] - m_all);
-            L = fmaf(wt[s], dsmem_ld_f32(dsmem_addr(a_l + (t * 128 + r) * 4, s)), L);
-          }
-        }
-        float acc[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-#pragma unroll
-        for (int s = 0; s < 8; ++s) {
-          if (s < S && wt[s] != 0.f) {
-            const uint32_t a = dsmem_addr(a_stg + ((t * D + cg * 32) * 128 + r) * 4, s);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] = fmaf(wt[s], dsmem_ld_f32(a + i * 512), acc[i]);
-          }
-        }
-        const float inv = 1.f / L;
-        __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D + cg * 32;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 vv;
-          vv.x = pack_bf16x2(acc[8 * i + 0] * inv, acc[8 * i + 1] * inv);
-          vv.y = pack_bf16x2(acc[8 * i + 2] * inv, acc[8 * i + 3] * inv);
-          vv.z = pack_bf16x2(acc[8 * i + 4] * inv, acc[8 * i + 5] * inv);
-          vv.w = pack_bf16x2(acc[8 * i + 6] * inv, acc[8 * i + 7] * inv);
-          reinterpret_cast<uint4*>(orow)[i] = vv;
-        }
-        if (cg == 0) {
-          float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
-          lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_all + log2f(L)) * 0.6931471805599453f;
-        }
-      }
-    }
-    cluster_arrive();                                         // nobody leaves while its shared memory is being read
-    cluster_wait();
-  }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 8) {

@@ -16,6 +16,7 @@
 #include "geom.cuh"
 #include "kernels_cc.cuh"
 #include "kernels_tc.cuh"
+#include "compress.cuh"
 
 using kvc::Geom;
 
@@ -348,6 +349,40 @@ static cudaError_t launch_tc2_attn(const Geom& g, const CUtensorMap& tq, const C
   kvc::attn_tc2_kernel<D><<<grid, 320, smem, st>>>(tq, tk, tv, (__nv_bfloat16*)out, (char*)ws, g);
   return cudaSuccess;
 }
+// a2..a4 fused (compress.cuh).  SCORE = false: the scores are already in the workspace.
+template <int D, bool SCORE>
+static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
+                                   int elem_bytes, cudaStream_t st) {
+  const int score_bytes = SCORE ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * 256 * 128 : 0;
+  const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4;
+  const int smem = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kvc::compress_kernel<D, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  // cluster size: spread one kv-head over several SMs when the heads alone cannot fill the GPU
+  // (about four key tiles per CTA: below that the two cluster barriers cost more than the tiles)
+  const int n_tiles = (g.n_cand + 127) / 128;
+  int Cn = (int)(kvc::kNumSMs / ((long long)g.Hkv * g.nl));
+  if (Cn > 8) Cn = 8;
+  if (Cn > (n_tiles + 3) / 4) Cn = (n_tiles + 3) / 4;
+  if (Cn < 1) Cn = 1;
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  lc.gridDim = dim3(Cn, g.Hkv, g.nl);
+  lc.blockDim = dim3(kvc::kCompressThreads, 1, 1);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = Cn; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kvc::compress_kernel<D, SCORE>, tk, tqo, (char*)cache, (char*)ws, g, Cn, elem_bytes);
+}
+
 template <int D>
 static cudaError_t launch_tc_score(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* ws,
                                    int tok_per_group, cudaStream_t st) {
@@ -461,31 +496,28 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (e != cudaSuccess) return check_cuda(c, e, "attention launch setup");
   c->launches++;
   if (evict) {
-    // a2 score
-    {
-    ProfScope ps(c, 2, st);
-    if (c->use_tc) {
-      e = D == 128 ? launch_tc_score<128>(g, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, tk, tqo, ws, tok_per_group, st);
-    } else if (f32) {
-      e = D == 128 ? launch_cc_score<float, 128>(g, q, cache, ws, st) : launch_cc_score<float, 64>(g, q, cache, ws, st);
-    } else {
-      e = D == 128 ? launch_cc_score<__nv_bfloat16, 128>(g, q, cache, ws, st) : launch_cc_score<__nv_bfloat16, 64>(g, q, cache, ws, st);
+    const bool fused_score = c->use_tc && g.w * g.G <= 256;    // observer rows fit one MMA: score inside the fused kernel
+    if (!fused_score) {
+      // a2 score as a kernel of its own (fp32 on CUDA cores; bf16 with more than 256 observer rows per kv-head)
+      ProfScope ps(c, 2, st);
+      if (c->use_tc) {
+        e = D == 128 ? launch_tc_score<128>(g, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, tk, tqo, ws, tok_per_group, st);
+      } else if (f32) {
+        e = D == 128 ? launch_cc_score<float, 128>(g, q, cache, ws, st) : launch_cc_score<float, 64>(g, q, cache, ws, st);
+      } else {
+        e = D == 128 ? launch_cc_score<__nv_bfloat16, 128>(g, q, cache, ws, st) : launch_cc_score<__nv_bfloat16, 64>(g, q, cache, ws, st);
+      }
+      if (e != cudaSuccess) return check_cuda(c, e, "score launch");
+      c->launches++;
     }
-    }
-    if (e != cudaSuccess) return check_cuda(c, e, "score launch setup");
-    c->launches++;
-    // a3 select
+    // (a2 +) a3 select + a4 compact
     {
       ProfScope ps(c, 3, st);
-      kvc::select_kernel<<<dim3(g.Hkv, 1, nl), 1024, 0, st>>>((const char*)cache, (char*)ws, g);
+      if (fused_score) e = D == 128 ? launch_compress<128, true>(g, tk, tqo, cache, ws, (int)c->elem, st)
+                                    : launch_compress<64, true>(g, tk, tqo, cache, ws, (int)c->elem, st);
+      else e = launch_compress<64, false>(g, tk, tk, cache, ws, (int)c->elem, st);
     }
-    c->launches++;
-    // a4 compact: at most min(n, tot - B) entries sit at or above row B
-    const int max_moves = n < g.tot - g.B ? n : g.tot - g.B;
-    {
-      ProfScope ps(c, 4, st);
-      kvc::compact_kernel<<<dim3((max_moves + 7) / 8, g.Hkv, nl), 256, 0, st>>>((char*)cache, (const char*)ws, g, (int)c->elem);
-    }
+    if (e != cudaSuccess) return check_cuda(c, e, "compress launch");
     c->launches++;
   }
   int rc = check_cuda(c, cudaGetLastError(), "kernel launch");

@@ -47,6 +47,9 @@ typedef enum { KVC_SCORE_ATTN = 0 /* query-aware score, Eq. 4 */ } kvc_policy;
 /* flags */
 #define KVC_FLAG_CUDA_CORES 1u /* bf16 only: run attention/score on the CUDA-core kernels used for
                                   fp32 instead of the tcgen05 tensor-core kernels (diagnostic) */
+#define KVC_FLAG_NO_KEY_SPLIT 4u /* attention: never split the key range over a thread-block cluster */
+#define KVC_FLAG_NO_PDL 8u     /* launch the kernels in plain stream order instead of letting each start
+                                  while its predecessor drains (programmatic dependent launch) */
 
 typedef struct {
   int n_layers;        /* L >= 1                                                                 */

@@ -107,6 +107,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
   int* mcount = reinterpret_cast<int*>(slot + p.mcount_off);
   volatile int* abort_flag = &sh.abort_flag;
   if (tid == 0) sh.abort_flag = 0;
+  pdl_launch_dependents();                        // the next kernel of the stream may set itself up meanwhile
 
   // ------------------------------------------------------------------------------------ phase 1: scores
   if constexpr (SCORE) {

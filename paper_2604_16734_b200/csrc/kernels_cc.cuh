@@ -2,6 +2,7 @@
 // (and, as a diagnostic, bf16 inputs).
 #pragma once
 #include "geom.cuh"
+#include "ptx.cuh"
 
 namespace kvc {
 
@@ -12,6 +13,8 @@ namespace kvc {
 template <typename T>
 __global__ void __launch_bounds__(256) append_kernel(const T* __restrict__ k, const T* __restrict__ v,
                                                      char* __restrict__ cache, Geom p) {
+  pdl_launch_dependents();                 // the attention kernel may set itself up meanwhile
+  pdl_wait();                              // the previous block's compaction still reads and writes this cache
   const int layer = blockIdx.z;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;

@@ -16,284 +16,12 @@ static constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 bf16 (one 128
 // kv-head.  A tile holds TOK = 128 / G tokens (TOK * G <= 128 rows).
 
 
-// ------------------------------------------------------------------------------------------------
-// a1 attention, two 128-row tiles (A, B) per CTA, software pipelined.
-//   warps 0-3  softmax of tile A     (thread = one row = one TMEM lane)
-//   warps 4-7  softmax of tile B
-//   warp  8    TMA producer: Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring of kStages
-//              32 KB slots
-//   warp  9    MMA issuer.  Issue order per key tile j:  O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ;
-//              O_B += P_B V_j ; S_B = Q_B K_{j+1}^T, so the tensor pipe works on one row tile while
-//              the CUDA cores run the softmax of the other.
-// TMEM columns: S_A/P_A [0,128)  S_B/P_B [128,256)  O_A [256,384)  O_B [384,512).
-// The running output is rescaled lazily: a row keeps its reference maximum until the true maximum
-// has grown by more than 2^8, so P stays below 256 and O rarely needs touching.
-// grid (ceil(ceil(n/TOK)/2), Hkv, nl), block 320, dynamic smem (2 + kStages) * (D/64) * 16 KB + 1 KB.
-static constexpr int kStages = 4;
-
-struct TcSmemAttn2 {
-  uint64_t q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_full[2], pv_done[2];
-  uint32_t tmem_base;
-  int abort_flag;
-};
-
-template <int D>
-__global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q,
-                                                          const __grid_constant__ CUtensorMap tm_k,
-                                                          const __grid_constant__ CUtensorMap tm_v,
-                                                          __nv_bfloat16* __restrict__ out, char* __restrict__ ws,
-                                                          Geom p) {
-  constexpr int NSUB = D / 64;
-  constexpr int TILE_BYTES = NSUB * kSubTileBytes;
-  constexpr uint32_t TMEM_COLS = 512;
-  constexpr float kRescaleThreshold = 8.f;      // log2 units
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;                            // two tiles
-  uint8_t* ring = smem + 2 * TILE_BYTES;         // kStages tiles
-  __shared__ TcSmemAttn2 sh;
-
-  const int layer = blockIdx.z, g = blockIdx.y;
-  const int TOK = 128 / p.G, rows = TOK * p.G;
-  const int tokA = blockIdx.x * 2 * TOK, tokB = tokA + TOK;
-  const bool has_B = tokB < p.n;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int last_tok = min(tokA + 2 * TOK, p.n) - 1;
-  const int kv_end = p.n_c + last_tok + 1;
-  const int T = (kv_end + 127) / 128;
-
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&sh.q_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.p_full[i], 128);
-      mbar_init(&sh.pv_done[i], 1);
-    }
-    for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
-    sh.abort_flag = 0;
-    mbar_fence_init();
-  }
-  // rows of the Q tiles that TMA never writes (rows >= TOK*G) must still be finite
-  {
-    const int pad16 = (128 - rows) * 8;          // 16-byte units per sub-tile
-    for (int i = threadIdx.x; i < 2 * NSUB * pad16; i += blockDim.x) {
-      const int sub = i / pad16, rem = i % pad16;
-      reinterpret_cast<uint4*>(sQ + sub * kSubTileBytes + rows * 128)[rem] = make_uint4(0, 0, 0, 0);
-    }
-  }
-  fence_proxy_async_smem();
-  if (warp == 8) {
-    tmem_alloc(&sh.tmem_base, TMEM_COLS);
-    tmem_relinquish();
-  }
-  tc_fence_before_sync();
-  __syncthreads();
-  tc_fence_after_sync();
-  const uint32_t tmem = sh.tmem_base;
-  volatile int* abort_flag = &sh.abort_flag;
-
-  if (warp == 8) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
-      mbar_expect_tx(&sh.q_full[0], NSUB * rows * 128);
-      for (int sub = 0; sub < NSUB; ++sub)
-        tma_load_4d(sQ + sub * kSubTileBytes, &tm_q, &sh.q_full[0], sub * 64, g * p.G, tokA, layer);
-      if (has_B) {
-        mbar_expect_tx(&sh.q_full[1], NSUB * rows * 128);
-        for (int sub = 0; sub < NSUB; ++sub)
-          tma_load_4d(sQ + TILE_BYTES + sub * kSubTileBytes, &tm_q, &sh.q_full[1], sub * 64, g * p.G, tokB, layer);
-      }
-      for (int i = 0; i < 2 * T; ++i) {          // item 2j = K_j, item 2j+1 = V_j
-        const int slot = i % kStages, round = i / kStages;
-        if (round > 0 && !mbar_wait(&sh.kv_empty[slot], (round - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(&sh.kv_full[slot], TILE_BYTES);
-        const CUtensorMap* tm = (i & 1) ? &tm_v : &tm_k;
-        for (int sub = 0; sub < NSUB; ++sub)
-          tma_load_4d(ring + slot * TILE_BYTES + sub * kSubTileBytes, tm, &sh.kv_full[slot], sub * 64, (i >> 1) * 128,
-                      g, layer);
-      }
-    }
-    __syncwarp();
-  } else if (warp == 9) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
-      const uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
-      const uint32_t aQ = smem_u32(sQ), aR = smem_u32(ring);
-      auto issue_S = [&](int t, int slot) {      // S_t = Q_t K^T, 16 of the d columns per MMA
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * kSubTileBytes + (kk % 4) * 32;
-          mma_ss(tmem + t * 128, smem_desc_sw128(aQ + t * TILE_BYTES + off, 16, 1024),
-                 smem_desc_sw128(aR + slot * TILE_BYTES + off, 16, 1024), idesc_qk, kk > 0);
-        }
-      };
-      auto issue_PV = [&](int t, int slot, bool acc) {   // O_t += P_t V, 16 keys per MMA
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
-                 smem_desc_sw128(aR + slot * TILE_BYTES + kk * 2048, kSubTileBytes, 1024), idesc_pv, acc || kk > 0);
-      };
-      bool ok = mbar_wait(&sh.q_full[0], 0, abort_flag) && mbar_wait(&sh.kv_full[0], 0, abort_flag);
-      if (ok) {
-        tc_fence_after_sync();
-        issue_S(0, 0);
-        mma_commit(&sh.s_full[0]);
-        if (has_B) {
-          ok = mbar_wait(&sh.q_full[1], 0, abort_flag);
-          if (ok) { issue_S(1, 0); mma_commit(&sh.s_full[1]); }
-        }
-        mma_commit(&sh.kv_empty[0]);
-      }
-      for (int j = 0; j < T && ok; ++j) {
-        const int iv = 2 * j + 1, ik = 2 * j + 2;
-        const int slotV = iv % kStages, slotK = ik % kStages;
-        const bool more = j + 1 < T;
-        ok = mbar_wait(&sh.p_full[0], j & 1, abort_flag) && mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after_sync();
-        issue_PV(0, slotV, j > 0);
-        mma_commit(&sh.pv_done[0]);
-        if (more) {
-          ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          issue_S(0, slotK);
-          mma_commit(&sh.s_full[0]);
-        }
-        if (has_B) {
-          ok = mbar_wait(&sh.p_full[1], j & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          issue_PV(1, slotV, j > 0);
-          mma_commit(&sh.pv_done[1]);
-        }
-        mma_commit(&sh.kv_empty[slotV]);
-        if (more) {
-          if (has_B) { issue_S(1, slotK); mma_commit(&sh.s_full[1]); }
-          mma_commit(&sh.kv_empty[slotK]);
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp < 4 || has_B) {
-    // ------------------------------------------------------------------ softmax + epilogue of tile t
-    const int t = warp >> 2;
-    const int r = (warp & 3) * 32 + lane;                     // row of the tile = TMEM lane
-    const int tok0 = t ? tokB : tokA;
-    const int tok = tok0 + r / p.G, hh = r % p.G;
-    const bool row_valid = r < rows && tok < p.n;
-    const int limit = p.n_c + tok + 1;                        // keys [0, limit) are visible to this row
-    const int tile_min_limit = p.n_c + tok0 + 1;              // smallest limit of any row of the tile
-    const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t tmem_S = tmem + t * 128 + lane_addr, tmem_O = tmem + 256 + t * 128 + lane_addr;
-    float m_ref = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < T; ++j) {
-      ok = mbar_wait(&sh.s_full[t], j & 1, abort_flag);
-      if (!ok) break;
-      tc_fence_after_sync();
-      uint32_t sr[128];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tmem_S + c * 32, sr + c * 32);
-      tmem_wait_ld();
-      if ((j + 1) * 128 > tile_min_limit) {                   // diagonal or tail tile: mask
-        const int lim = limit - j * 128;
-#pragma unroll
-        for (int c = 0; c < 128; ++c)
-          if (c >= lim) sr[c] = 0xff800000u;                  // -inf
-      }
-      float mx4[8];                                           // independent chains: latency, not issue, is the cost
-#pragma unroll
-      for (int i = 0; i < 8; ++i) mx4[i] = __uint_as_float(sr[i]);
-#pragma unroll
-      for (int c = 8; c < 128; c += 8) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sr[c + i]));
-      }
-      const float mx = fmaxf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])),
-                             fmaxf(fmaxf(mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
-      const float m_new = mx * p.scale_log2;                  // scale > 0
-      if (j == 0) {
-        m_ref = m_new == -INFINITY ? 0.f : m_new;
-      } else {
-        const bool grow = m_new > m_ref + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, grow)) {
-          const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;
-          if (grow) { m_ref = m_new; l *= f; }
-          ok = mbar_wait(&sh.pv_done[t], (j - 1) & 1, abort_flag);   // O_t holds every earlier tile
-          if (!ok) break;
-          tc_fence_after_sync();
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tmem_O + c * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-            tmem_st32(tmem_O + c * 32, o);
-          }
-        }
-      }
-      const float neg_m = -m_ref;
-      float ps[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i]), p.scale_log2, neg_m));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
-          ps[(i & 1) * 2] += p0;
-          ps[(i & 1) * 2 + 1] += p1;
-          pk[i] = pack_bf16x2(p0, p1);
-        }
-        tmem_st16(tmem_S + c * 16, pk);
-      }
-      l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(&sh.p_full[t]);
-    }
-    if (ok) ok = mbar_wait(&sh.pv_done[t], (T - 1) & 1, abort_flag);
-    if (ok) {
-      tc_fence_after_sync();
-      const float inv = 1.f / l;
-      __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tmem_O + c * 32, o);
-        tmem_wait_ld();
-        if (row_valid) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 vv;
-            vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-            vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-            vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-            vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-            reinterpret_cast<uint4*>(orow + c * 32)[i] = vv;
-          }
-        }
-      }
-      if (row_valid) {
-        float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
-        lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_ref + log2f(l)) * 0.6931471805599453f;
-      }
-    }
-  }
-  tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 8) {
-    tc_fence_after_sync();
-    tmem_dealloc(tmem, TMEM_COLS);
-  }
-  if (threadIdx.x == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
-}
+static constexpr int kStages = 4;                 // K/V ring slots of the attention kernel
 
 // ------------------------------------------------------------------------------------------------
-// a1 attention (Eq. 1): two 128-row tiles (A, B) per CTA, software pipelined, with the key range
-// optionally split over the CTAs of a thread-block cluster.
+// a0 + a1: append (Alg. 1) and attention (Eq. 1).  Two 128-row tiles (A, B) per CTA, software pipelined,
+// with the key range optionally split over the CTAs of a thread-block cluster.  Keys are the cache rows
+// [0, n_c) followed by the block's own tokens, which are read from the k/v inputs directly.
 //   warps 0-3   softmax of tile A     (thread = one row = one TMEM lane), 216 registers
 //   warps 4-7   softmax of tile B
 //   warp  8     TMA producer: Q tiles once, then K_j, V_j, K_j+1, ... through a ring of kStages 32 KB slots
@@ -302,6 +30,8 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
 //               (64 keys each) so the first PV MMAs start while the second half of the exponentials
 //               is still being computed.
 //   warp  11    only gives its registers away (setmaxnreg works on groups of four warps)
+// a0: before their first turn the threads of tile B copy the CTA's share of the block's keys, values and
+// positions into the cache.
 // The two softmax groups take turns (named barriers): while one tile's exponentials occupy the
 // CUDA cores the tensor pipe runs the other tile's MMAs; without the hand-over both tiles fall into
 // lockstep and the two pipes idle alternately.
@@ -318,16 +48,21 @@ __global__ void __launch_bounds__(320, 1) attn_tc2_kernel(const __grid_constant_
 // dynamic smem (2 + kStages) * (D/64) * 16 KB + 1 KB.
 static constexpr int kAttnThreads = 384;
 
-struct TcSmemAttn3 {
+struct TcSmemAttn {
   uint64_t q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_half[2][2], pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
 };
 
 template <int D>
-__global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_constant__ CUtensorMap tm_q,
+__global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                    const __grid_constant__ CUtensorMap tm_k,
                                                                    const __grid_constant__ CUtensorMap tm_v,
+                                                                   const __grid_constant__ CUtensorMap tm_kin,
+                                                                   const __grid_constant__ CUtensorMap tm_vin,
+                                                                   const __nv_bfloat16* __restrict__ k_in,
+                                                                   const __nv_bfloat16* __restrict__ v_in,
+                                                                   char* __restrict__ cache,
                                                                    __nv_bfloat16* __restrict__ out,
                                                                    char* __restrict__ ws, Geom p, int S) {
   constexpr int NSUB = D / 64;
@@ -338,7 +73,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;                            // two tiles
   uint8_t* ring = smem + 2 * TILE_BYTES;         // kStages tiles; after the key loop: the parked O tiles
-  __shared__ TcSmemAttn3 sh;
+  __shared__ TcSmemAttn sh;
 
   const int layer = blockIdx.z, g = blockIdx.y;
   const int split = S > 1 ? static_cast<int>(cluster_ctarank()) : 0;
@@ -348,11 +83,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
   const bool has_B = tokB < p.n;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int last_tok = min(tokA + 2 * TOK, p.n) - 1;
-  const int kv_end = p.n_c + last_tok + 1;
-  const int T = (kv_end + 127) / 128;            // key tiles this pair of row tiles can see
+  // Key tiles this pair of row tiles can see: Tc tiles of the cache (rows [0, n_c), the last one possibly
+  // partial), then the block's own keys in tiles of 128 tokens, read straight from the k/v inputs.
+  const int Tc = (p.n_c + 127) / 128;
+  const int T = Tc + (last_tok + 128) / 128;
   const int t_begin = split * T / S, t_end = (split + 1) * T / S;
   const int Tl = t_end - t_begin;                // key tiles of this CTA (0 is possible when S > T)
 
+  pdl_launch_dependents();                       // the next kernel of the stream may set itself up meanwhile
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.q_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.pv_done[i], 1);
@@ -388,6 +126,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
       // ---------------------------------------------------------------- TMA producer
       if (lane == 0) {
         tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_kin); tma_prefetch_desc(&tm_vin);
         pdl_wait();                                // the block's keys were appended by the previous kernel
       }
       if (lane == 0 && Tl > 0) {
@@ -403,10 +142,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
           const int slot = i % kStages, round = i / kStages;
           if (round > 0 && !mbar_wait(&sh.kv_empty[slot], (round - 1) & 1, abort_flag)) break;
           mbar_expect_tx(&sh.kv_full[slot], TILE_BYTES);
-          const CUtensorMap* tm = (i & 1) ? &tm_v : &tm_k;
-          for (int sub = 0; sub < NSUB; ++sub)
-            tma_load_4d(ring + slot * TILE_BYTES + sub * kSubTileBytes, tm, &sh.kv_full[slot], sub * 64,
-                        (t_begin + (i >> 1)) * 128, g, layer);
+          const int kt = t_begin + (i >> 1);
+          if (kt < Tc) {                           // cache rows kt*128 .. (rows past n_c are masked by the softmax)
+            const CUtensorMap* tm = (i & 1) ? &tm_v : &tm_k;
+            for (int sub = 0; sub < NSUB; ++sub)
+              tma_load_4d(ring + slot * TILE_BYTES + sub * kSubTileBytes, tm, &sh.kv_full[slot], sub * 64, kt * 128, g, layer);
+          } else {                                 // block tokens (kt - Tc)*128 .. (tokens past n are zero-filled)
+            const CUtensorMap* tm = (i & 1) ? &tm_vin : &tm_kin;
+            for (int sub = 0; sub < NSUB; ++sub)
+              tma_load_4d(ring + slot * TILE_BYTES + sub * kSubTileBytes, tm, &sh.kv_full[slot], sub * 64, g, (kt - Tc) * 128, layer);
+          }
         }
       }
     } else if (warp == 9 || (warp == 10 && has_B)) {
@@ -479,13 +224,45 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
     const int tok0 = t ? tokB : tokA;
     const int tok = tok0 + r / p.G, hh = r % p.G;
     const bool row_valid = r < rows && tok < p.n;
-    const int limit = p.n_c + tok + 1;                        // keys [0, limit) are visible to this row
-    const int tile_min_limit = p.n_c + tok0 + 1;              // smallest limit of any row of the tile
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tmem_S = tmem + t * 128 + lane_addr, tmem_O = tmem + 256 + t * 128 + lane_addr;
     float m_ref = -INFINITY, l = 0.f;                        // reference maximum (log2 units) and row sum
     bool ok = true;
     const bool active = t == 0 || has_B;
+    if (t == 1) {
+      // ---------------------------------------------------------------- a0 append (Alg. 1: C <- C u (K_i, V_i))
+      // Nobody in this kernel reads the appended rows (the block's keys come from the inputs), so the 128
+      // threads of tile B -- idle until tile A has had its first turn, or for the whole kernel when there
+      // is no tile B -- copy this CTA's share of the block's keys, values and positions into cache rows
+      // n_c .. tot.  The CTAs of a kv-head share the rows.
+      pdl_wait();                                            // the previous block's compaction is done with the cache
+      char* blob = cache + layer * p.cache_ls;
+      constexpr int VEC = D * 2 / 16;                        // 16-byte pieces per row (K or V)
+      constexpr int RPS = 128 / (2 * VEC);                   // rows per step of the 128 threads
+      constexpr int UNROLL = 4;                              // loads in flight per thread
+      const int sub = (threadIdx.x - 128) / (2 * VEC), piece = threadIdx.x % (2 * VEC);
+      const bool is_v = piece >= VEC;
+      const __nv_bfloat16* src_base = (is_v ? v_in : k_in) + layer * p.kv_ls;
+      char* dst_base = blob + (is_v ? p.v_off : 0);
+      const int stride = gridDim.x * RPS;
+      for (int t0 = blockIdx.x * RPS + sub; t0 < p.n; t0 += stride * UNROLL) {
+        uint4 val[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          const int tk = t0 + u * stride;
+          if (tk < p.n) val[u] = reinterpret_cast<const uint4*>(src_base + (static_cast<long long>(tk) * p.Hkv + g) * D)[piece % VEC];
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          const int tk = t0 + u * stride;
+          if (tk < p.n) {
+            const long long dst_row = static_cast<long long>(g) * p.cap + p.n_c + tk;
+            reinterpret_cast<uint4*>(dst_base + dst_row * D * 2)[piece % VEC] = val[u];
+            if (piece == 0) reinterpret_cast<int*>(blob + p.pos_off)[dst_row] = static_cast<int>(p.pos0 + tk);
+          }
+        }
+      }
+    }
     // Turn taking (named barrier 2 + t = "tile t may go", 128 waiters + 128 arrivals).  Tile A goes first.
     const bool turns = has_B && Tl > 0;
     if (turns && t == 1) named_barrier_arrive(2, 256);
@@ -502,8 +279,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc3_kernel(const __grid_
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tmem_S + c * 32, sr + c * 32);
         tmem_wait_ld();
-        if ((kt + 1) * 128 > tile_min_limit) {                // diagonal or tail tile: mask
-          const int lim = limit - kt * 128;
+        // columns [0, lim) of this tile are visible: a cache tile ends at row n_c, a block tile at the row's
+        // own token (causal inside the block); only the last cache tile and diagonal tiles need the mask
+        const int u = kt - Tc;                                // >= 0: tile of the block's own tokens
+        const int lim = u < 0 ? p.n_c - kt * 128 : tok + 1 - u * 128;
+        if (u < 0 ? lim < 128 : (u + 1) * 128 > tok0 + 1) {
 #pragma unroll
           for (int c = 0; c < 128; ++c)
             if (c >= lim) sr[c] = 0xff800000u;                // -inf

@@ -295,13 +295,33 @@ static cudaError_t launch_cc_score(const Geom& g, const void* q, void* cache, vo
   return cudaSuccess;
 }
 
+// Launch attributes shared by the PDL-aware kernels: an optional cluster size and, unless disabled,
+// programmatic stream serialization (the kernel may start while its predecessor drains; it calls
+// griddepcontrol.wait before it touches anything the predecessor wrote or still reads).
+struct LaunchAttrs {
+  cudaLaunchAttribute at[2];
+  int n;
+  LaunchAttrs(int cluster_x, bool pdl) : n(0) {
+    if (cluster_x > 0) {
+      at[n].id = cudaLaunchAttributeClusterDimension;
+      at[n].val.clusterDim.x = cluster_x; at[n].val.clusterDim.y = 1; at[n].val.clusterDim.z = 1;
+      ++n;
+    }
+    if (pdl) {
+      at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      at[n].val.programmaticStreamSerializationAllowed = 1;
+      ++n;
+    }
+  }
+};
+
 // Number of CTAs the key range of one row-tile pair is split over (= cluster size): enough to put
 // a CTA on every SM when the row tiles alone cannot, never more than the key tiles available.
 static int attn_key_splits(const Geom& g) {
   const int TOK = 128 / g.G;
   const int pairs = ((g.n + TOK - 1) / TOK + 1) / 2;
   const long long base = (long long)pairs * g.Hkv * g.nl;
-  const int T = (g.tot + 127) / 128;
+  const int T = (g.n_c + 127) / 128 + (g.n + 127) / 128;
   int S = (int)(kvc::kNumSMs / base);
   if (S > 8) S = 8;                    // portable cluster size limit
   if (S > T) S = T;
@@ -309,12 +329,13 @@ static int attn_key_splits(const Geom& g) {
 }
 
 template <int D>
-static cudaError_t launch_tc3_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                   void* out, void* ws, int S, cudaStream_t st) {
+static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                  const CUtensorMap& tkin, const CUtensorMap& tvin, const void* k, const void* v, void* cache,
+                                  void* out, void* ws, int S, bool pdl, cudaStream_t st) {
   const int smem = (2 + kvc::kStages) * (D / 64) * kvc::kSubTileBytes + 1024;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc3_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -326,33 +347,16 @@ static cudaError_t launch_tc3_attn(const Geom& g, const CUtensorMap& tq, const C
   lc.blockDim = dim3(kvc::kAttnThreads, 1, 1);
   lc.dynamicSmemBytes = smem;
   lc.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = S; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  lc.attrs = at;
-  lc.numAttrs = 1;
-  return cudaLaunchKernelEx(&lc, kvc::attn_tc3_kernel<D>, tq, tk, tv, (__nv_bfloat16*)out, (char*)ws, g, S);
-}
-template <int D>
-static cudaError_t launch_tc2_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                   void* out, void* ws, cudaStream_t st) {
-  const int smem = (2 + kvc::kStages) * (D / 64) * kvc::kSubTileBytes + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
-  const int TOK = 128 / g.G;
-  const int row_tiles = (g.n + TOK - 1) / TOK;
-  dim3 grid((row_tiles + 1) / 2, g.Hkv, g.nl);
-  kvc::attn_tc2_kernel<D><<<grid, 320, smem, st>>>(tq, tk, tv, (__nv_bfloat16*)out, (char*)ws, g);
-  return cudaSuccess;
+  LaunchAttrs la(S, pdl);
+  lc.attrs = la.at;
+  lc.numAttrs = la.n;
+  return cudaLaunchKernelEx(&lc, kvc::attn_tc_kernel<D>, tq, tk, tv, tkin, tvin, (const __nv_bfloat16*)k,
+                            (const __nv_bfloat16*)v, (char*)cache, (__nv_bfloat16*)out, (char*)ws, g, S);
 }
 // a2..a4 fused (compress.cuh).  SCORE = false: the scores are already in the workspace.
 template <int D, bool SCORE>
 static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
-                                   int elem_bytes, cudaStream_t st) {
+                                   int elem_bytes, bool pdl, cudaStream_t st) {
   const int score_bytes = SCORE ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * 256 * 128 : 0;
   const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4;
   const int smem = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
@@ -375,11 +379,9 @@ static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const C
   lc.blockDim = dim3(kvc::kCompressThreads, 1, 1);
   lc.dynamicSmemBytes = smem;
   lc.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = Cn; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  lc.attrs = at;
-  lc.numAttrs = 1;
+  LaunchAttrs la(Cn, pdl);
+  lc.attrs = la.at;
+  lc.numAttrs = la.n;
   return cudaLaunchKernelEx(&lc, kvc::compress_kernel<D, SCORE>, tk, tqo, (char*)cache, (char*)ws, g, Cn, elem_bytes);
 }
 
@@ -447,7 +449,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   const int D = cf.head_dim;
 
   // tensor maps first: nothing is enqueued if an encode fails
-  CUtensorMap tq, tk, tv, tqo;
+  CUtensorMap tq, tk, tv, tqo, tkin, tvin;
   int tok_per_group = 0;
   if (c->use_tc) {
     int rc = get_encoder(c);
@@ -462,6 +464,12 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     const uint32_t kb[4] = {64, 128, 1, 1};
     if ((rc = make_map(c, &tk, cache, kd, ks, kb))) return rc;
     if ((rc = make_map(c, &tv, (char*)cache + c->v_off, kd, ks, kb))) return rc;
+    // the block's own keys / values, read in place: k, v are [n][Hkv][d]
+    const uint64_t id[4] = {(uint64_t)D, (uint64_t)g.Hkv, (uint64_t)n, (uint64_t)nl};
+    const uint64_t is[3] = {(uint64_t)D * 2, (uint64_t)g.Hkv * D * 2, (uint64_t)kv_ls * 2};
+    const uint32_t ib[4] = {64, 1, 128, 1};
+    if ((rc = make_map(c, &tkin, k, id, is, ib))) return rc;
+    if ((rc = make_map(c, &tvin, v, id, is, ib))) return rc;
     if (evict) {
       tok_per_group = 256 / g.G;
       if (tok_per_group > g.w) tok_per_group = g.w;
@@ -470,23 +478,29 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     }
   }
 
-  // a0 append
-  {
+  const bool pdl = !(cf.flags & 8u);                   // flag 8: plain stream order between the kernels (diagnostic)
+  cudaError_t e = cudaSuccess;
+  // a0 append (the tensor-core attention kernel appends by itself)
+  if (!c->use_tc) {
     ProfScope ps(c, 0, st);
     dim3 grid((n * g.Hkv + 7) / 8, 1, nl);
-    if (f32) kvc::append_kernel<float><<<grid, 256, 0, st>>>((const float*)k, (const float*)v, (char*)cache, g);
-    else kvc::append_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (char*)cache, g);
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    lc.gridDim = grid; lc.blockDim = dim3(256, 1, 1); lc.stream = st;
+    LaunchAttrs la(0, pdl);
+    lc.attrs = la.at; lc.numAttrs = la.n;
+    if (f32) e = cudaLaunchKernelEx(&lc, kvc::append_kernel<float>, (const float*)k, (const float*)v, (char*)cache, g);
+    else e = cudaLaunchKernelEx(&lc, kvc::append_kernel<__nv_bfloat16>, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (char*)cache, g);
     c->launches++;
   }
+  if (e != cudaSuccess) return check_cuda(c, e, "append launch");
   // a1 attention
-  cudaError_t e = cudaSuccess;
   {
   ProfScope ps(c, 1, st);
-  if (c->use_tc && (cf.flags & 2u)) {       // previous kernel (no key split), kept for comparison while the new one is validated
-    e = D == 128 ? launch_tc2_attn<128>(g, tq, tk, tv, out, ws, st) : launch_tc2_attn<64>(g, tq, tk, tv, out, ws, st);
-  } else if (c->use_tc) {
+  if (c->use_tc) {
     const int S = (cf.flags & 4u) ? 1 : attn_key_splits(g);
-    e = D == 128 ? launch_tc3_attn<128>(g, tq, tk, tv, out, ws, S, st) : launch_tc3_attn<64>(g, tq, tk, tv, out, ws, S, st);
+    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, tkin, tvin, k, v, cache, out, ws, S, pdl, st)
+                 : launch_tc_attn<64>(g, tq, tk, tv, tkin, tvin, k, v, cache, out, ws, S, pdl, st);
   } else if (f32) {
     if (D == 128) launch_cc_attn<float, 128>(g, q, cache, out, ws, st); else launch_cc_attn<float, 64>(g, q, cache, out, ws, st);
   } else {
@@ -513,9 +527,9 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     // (a2 +) a3 select + a4 compact
     {
       ProfScope ps(c, 3, st);
-      if (fused_score) e = D == 128 ? launch_compress<128, true>(g, tk, tqo, cache, ws, (int)c->elem, st)
-                                    : launch_compress<64, true>(g, tk, tqo, cache, ws, (int)c->elem, st);
-      else e = launch_compress<64, false>(g, tk, tk, cache, ws, (int)c->elem, st);
+      if (fused_score) e = D == 128 ? launch_compress<128, true>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st)
+                                    : launch_compress<64, true>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st);
+      else e = launch_compress<64, false>(g, tk, tk, cache, ws, (int)c->elem, pdl, st);
     }
     if (e != cudaSuccess) return check_cuda(c, e, "compress launch");
     c->launches++;

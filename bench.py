@@ -279,6 +279,21 @@ class Runner:
                 kv.prefill_chunk_host(l, qh[l, p:p + n], kh[l, p:p + n], vh[l, p:p + n], p, oh[l, p:p + n])
 
 
+def max_over_ranks(seconds: float, dist, device) -> float:
+    """The job is as slow as its slowest rank: MAX-reduce a duration over the process group (if any)."""
+    if dist is None:
+        return seconds
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_layer: int, layers: int, steps: int, world: int, seconds: float) -> float:
+    """Metric of the whole job: every rank runs a replica of the request (weak scaling), so the tokens x layers
+    all ranks processed in `steps` steps, divided by the time of the slowest rank."""
+    return world * tokens_per_layer * layers * steps / seconds
+
+
 def time_steps(fn, steps, barrier):
     barrier()
     torch.cuda.synchronize()
@@ -294,8 +309,9 @@ def time_steps(fn, steps, barrier):
     return e0.elapsed_time(e1) / 1e3, t0, t1
 
 
-def profile_pass(r: Runner, steps: int):
-    """Per-kernel CUDA-event durations (on the launching stream) and exact algorithmic work, direct calls."""
+def profile_pass(r: Runner, steps: int, batched: bool = False):
+    """Per-kernel CUDA-event durations (on the launching stream) and exact algorithmic work: one call per
+    (block, layer), or with `batched` one call per block with the layer index in the launch grid."""
     kv, cfg = r.kvc, r.cfg
     work = {s: dict(bytes=0, flops=0) for s in STEPS}
     # exact move counts need one pass with a readback after every call
@@ -307,14 +323,14 @@ def profile_pass(r: Runner, steps: int):
             kv._check(kv._lib.kvc_prefill_chunk(kv._h, l, q, k, v, n, p, kv.cache[l].data_ptr(), kv.workspace.data_ptr(),
                                                 o, kv._stream()))
             moves = kv.move_counts(0).tolist() if n_c + n > cfg.budget else None
-            fused = cfg.dtype == "bf16" and not (r.flags & 1) and min(cfg.obs_window, n) * cfg.group <= 256
+            fused = cfg.dtype == "bf16" and not (r.flags & 1) and min(cfg.obs_window, n) * cfg.group <= 128
             for s, wv in work_of_call(cfg, n, n_c, moves, fused).items():
                 work[s]["bytes"] += wv["bytes"]; work[s]["flops"] += wv["flops"]
         n_c = min(n_c + n, cfg.budget)
     torch.cuda.synchronize()
     kv.profile_enable(True)
     for _ in range(steps):
-        r.step_direct()
+        (r.step_batched if batched else r.step_direct)()
     torch.cuda.synchronize()
     ms, cnt = kv.profile_read()
     kv.profile_enable(False)
@@ -387,12 +403,9 @@ def main():
     if args.mode != "graph":
         launches_per_step = (kv.launch_count() - launches_before) // args.steps
     assert kv.status() == 0, kv.last_error()
-    if dist is not None:
-        t = torch.tensor([secs], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        secs = float(t.item())
+    secs = max_over_ranks(secs, dist, "cuda")
     tokens_layers = cfg.n_tokens * L
-    value = world * tokens_layers * args.steps / secs
+    value = whole_job_value(cfg.n_tokens, L, args.steps, world, secs)
 
     # ---- per-kernel durations and roofline (rank 0, outside the timed region)
     per, roof = {}, None
@@ -415,6 +428,17 @@ def main():
         roof["us_per_launch"] = d["us_per_launch"]
         roof["arithmetic_intensity"] = ai
 
+    # ---- the same kernels with all layers in one launch (possible only with synthetic inputs): what the
+    #      bandwidth-bound steps reach when a launch carries enough bytes to fill the GPU
+    per_b = {}
+    if rank == 0 and not args.no_profile and L > 1:
+        per_b = profile_pass(r, 3, batched=True)
+        for s, d in per_b.items():
+            sec = d["ms_total_per_step"] / 1e3
+            d["gbs"] = d["bytes_per_step"] / sec / 1e9
+            d["tflops"] = d["flops_per_step"] / sec / 1e12
+            d["hbm_frac"] = d["gbs"] / peaks["hbm_gbs"]
+
     # ---- end to end through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
@@ -424,10 +448,7 @@ def main():
         torch.cuda.synchronize()
         e_steps = max(1, min(args.steps, 5))
         esecs, _, _ = time_steps(lambda: r.step_host(host), e_steps, barrier)
-        if dist is not None:
-            t = torch.tensor([esecs], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            esecs = float(t.item())
+        esecs = max_over_ranks(esecs, dist, "cuda")
         h2d = sum(t.numel() * t.element_size() for t in host[:3])
         d2h = host[3].numel() * host[3].element_size()
         e2e = dict(value=world * tokens_layers * e_steps / esecs, unit=UNIT, h2d_bytes_per_step=h2d,
@@ -460,7 +481,7 @@ def main():
                 "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
                 "kv_bytes": {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,
                              "blobs_incl_positions": kv.blob_bytes * L},
-                "kernels": per}
+                "kernels": per, "kernels_layer_batched": per_b}
         if roof:
             line["roofline"] = roof
         if e2e:

@@ -15,7 +15,7 @@
 // Entry j gets the key (score bits << 32) | ~pos: a larger key means a higher score and, at equal
 // score, an older entry; keys are unique because positions are.  Scores are sums of probabilities,
 // hence >= 0, so their IEEE bit patterns order like integers.  The n_keep-th largest key (the cut-off)
-// is found exactly by an MSB-first radix descent with 12-bit digits that starts below the bits all
+// is found exactly by an MSB-first radix descent with 11-bit digits that starts below the bits all
 // keys share and stops as soon as the bin that holds the cut-off survives as a whole.
 #pragma once
 #include <cuda.h>
@@ -24,10 +24,14 @@
 
 namespace kvc {
 
-static constexpr int kCompressThreads = 1024;
-static constexpr int kSelBins = 4096;
-static constexpr int kMaxKeysSmem = 8192;     // candidates whose keys fit the shared-memory table (64 KB)
-static constexpr int kMaxMovesSmem = 4096;    // moves whose (src, dst) fit the shared-memory tables (32 KB)
+// 512 threads and at most ~108 KB of shared memory per CTA: two CTAs share an SM, so that one scores
+// (TMA / tensor-core bound) while the other selects (barrier bound) when many kv-heads are in flight.
+static constexpr int kCompressThreads = 512;
+static constexpr int kDigitBits = 11;
+static constexpr int kSelBins = 1 << kDigitBits;
+static constexpr int kMaxKeysSmem = 6144;     // candidates whose keys fit the shared-memory table (48 KB)
+static constexpr int kMaxMovesSmem = 2048;    // moves whose (src, dst) fit the shared-memory tables (16 KB)
+static constexpr int kMaxObsRowsFused = 128;  // observer rows (w * G) the fused scoring phase takes
 static constexpr int kSubTileBytesC = 128 * 128;
 
 __device__ __forceinline__ unsigned long long select_key(float score, int pos) {
@@ -35,14 +39,14 @@ __device__ __forceinline__ unsigned long long select_key(float score, int pos) {
          static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(pos));
 }
 
-// The selection and the listing run on a team of kTeam threads (measured: a smaller team pays less per
-// barrier but more per key, and loses; the whole block it is).
+// The selection and the listing run on a team of kTeam threads: the whole block (measured: a quarter of
+// it pays less per barrier but more per key, and loses).
 static constexpr int kTeam = kCompressThreads;
 __device__ __forceinline__ void team_sync() { named_barrier(3, kTeam); }
 
 // Inclusive scan of one int per team thread; returns the inclusive value and the team total.
 // scratch: kTeam / 32 + 1 ints of shared memory.  Only warp 0 combines the warp totals: a value that
-// every thread reads costs one load per warp, 32 of them cost 1024.
+// every thread reads costs one load per warp, so 16 such values would cost 256 loads.
 __device__ __forceinline__ int team_scan_incl(int v, int* scratch, int* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int incl = v;
@@ -55,17 +59,17 @@ __device__ __forceinline__ int team_scan_incl(int v, int* scratch, int* total) {
   if (lane == 31) scratch[warp] = incl;
   team_sync();
   if (warp == 0) {
-    int t = scratch[lane], ti = t;
+    int t = lane < kTeam / 32 ? scratch[lane] : 0, ti = t;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int y = __shfl_up_sync(0xffffffffu, ti, o);
       if (lane >= o) ti += y;
     }
-    scratch[lane] = ti - t;               // exclusive warp offsets
-    if (lane == 31) scratch[32] = ti;
+    if (lane < kTeam / 32) scratch[lane] = ti - t;   // exclusive warp offsets
+    if (lane == 31) scratch[kTeam / 32] = ti;
   }
   team_sync();
-  *total = scratch[32];
+  *total = scratch[kTeam / 32];
   return incl + scratch[warp];
 }
 
@@ -81,16 +85,17 @@ struct CompressSmem {
   int s_remaining, s_bin_count;
 };
 
-// grid (Cn, Hkv, nl), cluster (Cn,1,1), block 1024.
-// dynamic smem: SCORE ? 2 * (D/64) * 16 KB + (D/64) * 32 KB + 1 KB : 96 KB + 1 KB (key and move tables).
+// grid (Cn, Hkv, nl), cluster (Cn,1,1), block 512.
+// dynamic smem: the larger of the scoring buffers (two K tiles + up to 128 observer rows) and of the key
+// and move tables (64 KB), + 1 KB.
 template <int D, bool SCORE>
-__global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __grid_constant__ CUtensorMap tm_k,
+__global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __grid_constant__ CUtensorMap tm_k,
                                                                        const __grid_constant__ CUtensorMap tm_qobs,
                                                                        char* __restrict__ cache, char* __restrict__ ws,
                                                                        Geom p, int Cn, int elem_bytes) {
   constexpr int NSUB = D / 64;
   constexpr int K_TILE_BYTES = NSUB * kSubTileBytesC;
-  constexpr int kQSubBytes = 256 * 128;          // up to 256 observer rows x 128 B
+  constexpr int kQSubBytes = kMaxObsRowsFused * 128;   // up to 128 observer rows x 128 B
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ CompressSmem sh;
@@ -115,7 +120,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
     uint8_t* sQ = smem + 2 * K_TILE_BYTES;           // observer rows
     const int n_tiles = (p.n_cand + 127) / 128;
     const int my_tiles = rank < n_tiles ? (n_tiles - rank + Cn - 1) / Cn : 0;
-    const int cols = p.w * p.G;                      // observer columns (<= 256: one MMA group)
+    const int cols = p.w * p.G;                      // observer columns (<= 128: one MMA, two accumulators of 128 columns)
     const int n_mma = (cols + 15) & ~15;
     if (tid == 0) {
       mbar_init(&sh.q_full, 1);
@@ -126,7 +131,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
     for (int i = tid; i < NSUB * kQSubBytes / 16; i += kCompressThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     if (warp == 8) {
-      tmem_alloc(&sh.tmem_base, 512);
+      tmem_alloc(&sh.tmem_base, 256);
       tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -161,7 +166,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
           tc_fence_after_sync();
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk)
-            mma_ss_lh(tmem + b * 256, k_lo0 + ((b * K_TILE_BYTES + (kk / 4) * kSubTileBytesC + (kk % 4) * 32) >> 4), hi,
+            mma_ss_lh(tmem + b * 128, k_lo0 + ((b * K_TILE_BYTES + (kk / 4) * kSubTileBytesC + (kk % 4) * 32) >> 4), hi,
                       q_lo + (((kk / 4) * kQSubBytes + (kk % 4) * 32) >> 4), hi, idesc, kk > 0);
           mma_commit(&sh.s_full[b]);
           if (i + 2 < my_tiles) {                    // refill K buffer b once the MMAs that read it are done
@@ -198,8 +203,8 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
         for (int c0 = 0; c0 < n_mma; c0 += 32) {       // n_mma is a multiple of 16: the second half may be absent
           uint32_t sr[32];
           const bool two = c0 + 16 < n_mma;
-          tmem_ld16(tmem + b * 256 + lane_addr + c0, sr);
-          if (two) tmem_ld16(tmem + b * 256 + lane_addr + c0 + 16, sr + 16);
+          tmem_ld16(tmem + b * 128 + lane_addr + c0, sr);
+          if (two) tmem_ld16(tmem + b * 128 + lane_addr + c0 + 16, sr + 16);
           tmem_wait_ld();
 #pragma unroll
           for (int k = 0; k < 16; ++k) acc += fast_exp2(fmaf(__uint_as_float(sr[k]), p.scale_log2, -sh.lse2[c0 + k]));
@@ -219,7 +224,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
     __syncthreads();
     if (warp == 8) {
       tc_fence_after_sync();
-      tmem_dealloc(tmem, 512);
+      tmem_dealloc(tmem, 256);
     }
   } else {
     if (tid == 0) pdl_wait();
@@ -233,9 +238,9 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
   }
 
   // ------------------------------------------------------------------------------------ phase 2: selection
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);           // 64 KB
-  int* tab_src = reinterpret_cast<int*>(smem + kMaxKeysSmem * 8);                    // 16 KB
-  int* tab_dst = tab_src + kMaxMovesSmem;                                            // 16 KB
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);           // 48 KB
+  int* tab_src = reinterpret_cast<int*>(smem + kMaxKeysSmem * 8);                    // 8 KB
+  int* tab_dst = tab_src + kMaxMovesSmem;                                            // 8 KB
   const bool keys_in_smem = p.n_cand <= kMaxKeysSmem;
   if (keys_in_smem)
     for (int j = tid; j < p.n_cand; j += kCompressThreads) keys[j] = select_key(__ldcg(score + j), pos[j]);
@@ -256,7 +261,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
       if (lane == 0) { sh.list[warp] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[kTeam / 32 + warp] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
       team_sync();
       if (warp == 0) {                                           // one warp folds the 32 partial results
-        const unsigned long long pa = sh.list[lane], po = sh.list[kTeam / 32 + lane];
+        const unsigned long long pa = lane < kTeam / 32 ? sh.list[lane] : ~0ull, po = lane < kTeam / 32 ? sh.list[kTeam / 32 + lane] : 0ull;
         a_lo = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(pa)); a_hi = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(pa >> 32));
         o_lo = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(po)); o_hi = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(po >> 32));
         if (lane == 0) { sh.list[2 * (kTeam / 32)] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[2 * (kTeam / 32) + 1] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
@@ -265,7 +270,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
       k_and = sh.list[2 * (kTeam / 32)]; k_or = sh.list[2 * (kTeam / 32) + 1];
       const unsigned long long differ = k_and ^ k_or;           // != 0: at least two distinct keys (n_cand > n_keep >= 1)
       const int top = 63 - __clzll(static_cast<long long>(differ));
-      int shift = top >= 11 ? top - 11 : 0, bits = top - shift + 1;
+      int shift = top >= kDigitBits - 1 ? top - (kDigitBits - 1) : 0, bits = top - shift + 1;
       team_sync();                                               // sh.list is reused below
       if (tid == 0) { sh.s_prefix = top == 63 ? 0ull : (k_or >> (top + 1)) << (top + 1); sh.s_remaining = p.n_keep; }
       while (true) {
@@ -279,7 +284,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
           if (hi >= 64 || (key >> hi) == (prefix >> hi)) atomicAdd(&sh.hist[(key >> shift) & ((1u << bits) - 1)], 1);
         }
         team_sync();
-        // descending scan: thread t owns the BPT bins from 4095 - BPT*t downwards
+        // descending scan: thread t owns the BPT bins from kSelBins - 1 - BPT*t downwards
         constexpr int BPT = kSelBins / kTeam;
         const int b0 = kSelBins - 1 - BPT * tid;
         int mine = 0;
@@ -299,7 +304,7 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
         // Done when every bit is decided, or when the whole bin survives (its rank equals its size): then
         // the prefix with zeros below it separates the retained keys from the others.
         if (shift == 0 || sh.s_remaining == sh.s_bin_count) break;
-        bits = shift >= 12 ? 12 : shift;
+        bits = shift >= kDigitBits ? kDigitBits : shift;
         shift -= bits;
       }
     }
@@ -318,9 +323,9 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
   {
     // Each warp owns a contiguous segment of the rows, walked 32 rows at a time (lane = row, so the
     // shared-memory keys are read without bank conflicts).  Pass 1 counts the warp's holes (rows below
-    // B) and survivors (rows from B on), one scan over the 32 warps turns the counts into offsets,
+    // B) and survivors (rows from B on), one scan over the warps turns the counts into offsets,
     // pass 2 writes the row indices in ascending order.
-    const int seg = ((p.tot + 31) / 32 + 31) & ~31;              // rows per warp, a multiple of 32
+    const int seg = ((p.tot + kTeam / 32 - 1) / (kTeam / 32) + 31) & ~31;   // rows per warp, a multiple of 32
     const int s0 = warp * seg, s1 = min(s0 + seg, p.tot);
     auto retained = [&](int j) { return j >= p.n_cand || key_of(j) >= thr; };
     int holes = 0, surv = 0;
@@ -372,17 +377,35 @@ __global__ void __launch_bounds__(kCompressThreads, 1) compress_kernel(const __g
   const long long row_bytes = static_cast<long long>(p.d) * elem_bytes;
   const int vec = static_cast<int>(row_bytes / 16);
   const long long head = static_cast<long long>(g) * p.cap;
-  for (int mv = rank * (kCompressThreads / 32) + warp; mv < total_holes; mv += Cn * (kCompressThreads / 32)) {
-    const int src = msrc[mv], dst = mdst[mv];
-    const uint4* ks = reinterpret_cast<const uint4*>(blob + (head + src) * row_bytes);
-    const uint4* vs = reinterpret_cast<const uint4*>(blob + p.v_off + (head + src) * row_bytes);
-    uint4* kd = reinterpret_cast<uint4*>(blob + (head + dst) * row_bytes);
-    uint4* vd = reinterpret_cast<uint4*>(blob + p.v_off + (head + dst) * row_bytes);
-    for (int i = lane; i < 2 * vec; i += 32) {
-      if (i < vec) kd[i] = ks[i];
-      else vd[i - vec] = vs[i - vec];
+  // (row = 2 * vec pieces of 16 bytes, K then V; a warp keeps kMovesInFlight moves in flight, since one
+  // load-then-store at a time would leave the copy latency-bound)
+  constexpr int kMovesInFlight = 4;
+  const int wstride = Cn * (kCompressThreads / 32);
+  for (int mv0 = rank * (kCompressThreads / 32) + warp; mv0 < total_holes; mv0 += wstride * kMovesInFlight) {
+    int src[kMovesInFlight], dst[kMovesInFlight];
+#pragma unroll
+    for (int u = 0; u < kMovesInFlight; ++u) {
+      const int mv = mv0 + u * wstride;
+      src[u] = mv < total_holes ? msrc[mv] : -1;
+      dst[u] = mv < total_holes ? mdst[mv] : -1;
     }
-    if (lane == 0) pos[dst] = pos[src];
+    for (int i = lane; i < 2 * vec; i += 32) {
+      const long long off = (i < vec ? 0 : p.v_off) + static_cast<long long>(i < vec ? i : i - vec) * 16;
+      uint4 val[kMovesInFlight];
+#pragma unroll
+      for (int u = 0; u < kMovesInFlight; ++u)
+        if (src[u] >= 0) val[u] = *reinterpret_cast<const uint4*>(blob + off + (head + src[u]) * row_bytes);
+#pragma unroll
+      for (int u = 0; u < kMovesInFlight; ++u)
+        if (src[u] >= 0) *reinterpret_cast<uint4*>(blob + off + (head + dst[u]) * row_bytes) = val[u];
+    }
+    if (lane < kMovesInFlight && src[0] >= 0) {
+      int sj = -1, dj = -1;
+#pragma unroll
+      for (int u = 0; u < kMovesInFlight; ++u)
+        if (lane == u) { sj = src[u]; dj = dst[u]; }
+      if (sj >= 0) pos[dj] = pos[sj];
+    }
   }
   if (tid == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
 }

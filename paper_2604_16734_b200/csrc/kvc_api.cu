@@ -357,12 +357,13 @@ static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CU
 template <int D, bool SCORE>
 static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
                                    int elem_bytes, bool pdl, cudaStream_t st) {
-  const int score_bytes = SCORE ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * 256 * 128 : 0;
+  const int score_bytes = SCORE ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * kvc::kMaxObsRowsFused * 128 : 0;
   const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4;
-  const int smem = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
+  const int smem_min = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
+  const int smem_solo = 120 * 1024;                      // more than half an SM: one CTA per SM
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::compress_kernel<D, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(kvc::compress_kernel<D, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_solo);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -373,6 +374,10 @@ static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const C
   if (Cn > 8) Cn = 8;
   if (Cn > (n_tiles + 3) / 4) Cn = (n_tiles + 3) / 4;
   if (Cn < 1) Cn = 1;
+  // Two CTAs share an SM only when there are more CTAs than SMs (then one scores while the other selects);
+  // a launch that fits the GPU asks for more than half an SM's shared memory so that every CTA gets an SM
+  // of its own instead of being packed in pairs.
+  const int smem = (long long)Cn * g.Hkv * g.nl > kvc::kNumSMs ? smem_min : smem_solo;
   cudaLaunchConfig_t lc;
   memset(&lc, 0, sizeof(lc));
   lc.gridDim = dim3(Cn, g.Hkv, g.nl);
@@ -510,9 +515,9 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (e != cudaSuccess) return check_cuda(c, e, "attention launch setup");
   c->launches++;
   if (evict) {
-    const bool fused_score = c->use_tc && g.w * g.G <= 256;    // observer rows fit one MMA: score inside the fused kernel
+    const bool fused_score = c->use_tc && g.w * g.G <= kvc::kMaxObsRowsFused;   // few observer rows: score inside the fused kernel
     if (!fused_score) {
-      // a2 score as a kernel of its own (fp32 on CUDA cores; bf16 with more than 256 observer rows per kv-head)
+      // a2 score as a kernel of its own (fp32 on CUDA cores; bf16 with more than 128 observer rows per kv-head)
       ProfScope ps(c, 2, st);
       if (c->use_tc) {
         e = D == 128 ? launch_tc_score<128>(g, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, tk, tqo, ws, tok_per_group, st);

@@ -71,6 +71,24 @@ def test_c5_long_video_blocks():
 
 
 # ------------------------------------------------------------------------------------------------
+# the benchmark's configurations at FULL size (every block of the whole prefix, the launch geometry the
+# benchmark times: one layer per call), checked on the kv-heads the oracle can follow in reasonable time
+
+@pytest.mark.parametrize("name,kv_heads", [("C2", None), ("C3", None), ("C4", [0, 5]), ("C5", [3])])
+def test_full_size_one_layer(name, kv_heads):
+    cfg = reduced(CONFIGS[name], n_layers=1)
+    kvc = _kvc_for(cfg)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=kv_heads)
+    assert worst["err_out"] <= 2e-2
+    # the cache never exceeds the budget, and ends exactly at it once the prefix is longer than B
+    K, V, pos, ln = kvc.cache_view(0)
+    assert ln == min(cfg.n_tokens, cfg.budget)
+    for g in range(cfg.n_kv_heads):
+        kept = pos[g, :ln].tolist()
+        assert len(set(kept)) == ln and min(kept) >= 0 and max(kept) == cfg.n_tokens - 1
+
+
+# ------------------------------------------------------------------------------------------------
 # ragged shapes and degenerate cases
 
 @pytest.mark.parametrize("dtype,d,hq,hkv,flags", [

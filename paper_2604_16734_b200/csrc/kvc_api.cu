@@ -316,7 +316,10 @@ struct LaunchAttrs {
 };
 
 // Number of CTAs the key range of one row-tile pair is split over (= cluster size): enough to put
-// a CTA on every SM when the row tiles alone cannot, never more than the key tiles available.
+// a CTA on every SM when the row tiles alone cannot, as long as every CTA keeps a few key tiles.
+// (An exchange of the partials through an L2-resident global buffer instead of distributed shared
+// memory was measured too: slower, the release / acquire round trip costs more than the narrow
+// SM-to-SM path.)
 static int attn_key_splits(const Geom& g) {
   const int TOK = 128 / g.G;
   const int pairs = ((g.n + TOK - 1) / TOK + 1) / 2;
@@ -324,7 +327,7 @@ static int attn_key_splits(const Geom& g) {
   const int T = (g.n_c + 127) / 128 + (g.n + 127) / 128;
   int S = (int)(kvc::kNumSMs / base);
   if (S > 8) S = 8;                    // portable cluster size limit
-  if (S > T) S = T;
+  if (S > T / 3) S = T / 3;            // the exchange costs about as much as two key tiles: keep three per CTA
   return S < 1 ? 1 : S;
 }
 

@@ -52,6 +52,34 @@ def load_peaks():
 
 
 # ------------------------------------------------------------------------------------------------
+# DRAM traffic of one steady-state launch (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture,
+# summarised under profiles/), valid only for the kernel sources it was taken from: the hash below is that
+# of the CUDA sources at capture time, and the figure is reported as null once they have changed.
+
+NCU_TRAFFIC = {
+    "sources": "c24fe5b5f95ff980",
+    "bytes_per_launch": {("C2", "attention"): 7409664, ("C2", "compress"): 4203264,
+                         ("C5", "attention"): 29439488, ("C5", "compress"): 12477696},
+}
+
+
+def kernel_sources_hash():
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2604_16734_b200", "csrc", "*"))):
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload, kernel):
+    if kernel_sources_hash() != NCU_TRAFFIC["sources"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"].get((workload, kernel))
+
+
+# ------------------------------------------------------------------------------------------------
 # algorithmic work of one launch (what the method itself has to move / compute)
 
 def work_of_call(cfg, n, n_c, moves_per_head=None, fused_score=True):
@@ -387,7 +415,7 @@ def main():
     sampler.start()
 
     step = {"direct": r.step_direct, "batched": r.step_batched, "graph": r.step_graph}[args.mode]
-    r.step_direct()                       # sets function attributes, resolves the driver entry point
+    (r.step_batched if args.mode == "batched" else r.step_direct)()   # sets function attributes, resolves the driver entry point
     torch.cuda.synchronize()
     if args.mode == "graph":
         r.capture()
@@ -425,6 +453,8 @@ def main():
         else:
             roof = dict(kernel=dom, bound="hbm", achieved=d["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
                         frac=d["gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"])
+        roof["traffic"] = ncu_traffic(cfg.name, dom) if L == cfg.n_layers else None
+        roof["algorithmic_bytes_per_launch"] = d["bytes_per_step"] / max(d["launches_per_step"], 1)
         roof["us_per_launch"] = d["us_per_launch"]
         roof["arithmetic_intensity"] = ai
 

@@ -26,7 +26,12 @@ design notes of the repository):
   * the probabilities are the true attention probabilities of those rows, i.e.
     normalised over everything the row attends to;
   * ties at the cut-off keep the older entry (smaller position);
-  * scores are recomputed from scratch at every eviction round.
+  * scores are recomputed from scratch at every eviction round;
+  * query-agnostic policy (Sec. 3.2, "Query-Agnostic Eviction"): the anchor mu is the mean of the
+    raw keys the cache holds right after the block was appended, "similarity" is the cosine, and
+    the score of an entry is 1 - cos(k_j, mu) (so "lower similarity" = higher score = retained);
+    the same last-w entries are protected and ties keep the older entry; a zero key or a zero
+    anchor has cosine 0.
 
 Pins (tests/test_oracle_pins.py): budget >= sequence length reproduces dense
 causal attention (library routine); empty-cache block equals causal attention
@@ -34,7 +39,9 @@ on the block; permutation invariance over cache order; probability mass of the
 score; one observer / one head reduces to a single softmax row; one block of
 the whole sequence reproduces post-prefill compression computed with library
 softmax / top-k; brute-force subset enumeration on tiny inputs; tie-break on
-duplicated keys; retained rows are bit-identical copies; Eq. 2 byte counts.
+duplicated keys; retained rows are bit-identical copies; Eq. 2 byte counts.  Query-agnostic
+score: library cosine similarity; an outlier among identical keys is the one kept; invariance
+under a common scaling and a common rotation of all keys; brute force.
 End-to-end model accuracy (the paper's tables): parity unpinned, it needs
 datasets and weights that are not available.
 """
@@ -61,12 +68,14 @@ class KVCOracle:
     """Budgeted KV cache of one model: state is, per (layer, kv-head), a list of (pos, k, v)."""
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
-                 budget: int, obs_window: int = 32, scale: Optional[float] = None):
+                 budget: int, obs_window: int = 32, scale: Optional[float] = None, policy: str = "attn"):
         assert n_q_heads % n_kv_heads == 0
         self.L, self.Hq, self.Hkv, self.d = n_layers, n_q_heads, n_kv_heads, head_dim
         self.G = n_q_heads // n_kv_heads
         self.M = budget
         self.obs_window = obs_window
+        assert policy in ("attn", "keydiff")
+        self.policy = policy
         self.scale = (1.0 / np.sqrt(head_dim)) if scale is None else float(scale)   # Eq. 1: 1/sqrt(d_k)
         self.reset()
 
@@ -152,7 +161,14 @@ class KVCOracle:
             w = min(self.obs_window, n)
             assert w <= M
             n_cand = tot - w
-            score = P[:, n - w:, :n_cand].sum(axis=(0, 1))
+            if self.policy == "attn":
+                score = P[:, n - w:, :n_cand].sum(axis=(0, 1))
+            else:
+                # query-agnostic (Sec. 3.2): anchor = mean of the cached keys, keep the keys least similar to it
+                mu = K.mean(axis=0)
+                denom = np.linalg.norm(K[:n_cand], axis=1) * np.linalg.norm(mu)
+                cos = np.divide(K[:n_cand] @ mu, denom, out=np.zeros(n_cand), where=denom > 0)
+                score = 1.0 - cos
 
             # 4. select: keep the (M - w) candidates that come first under
             #    (score descending, position ascending); evict the other tot - M (Alg. 1)

@@ -274,3 +274,72 @@ def test_planted_mistakes_are_caught():
     # transposed operand: swapping k and v must not reproduce the reference
     out, _ = _run_chunks(KVCOracle(1, 2, 1, 8, budget=64), q, v, k, [12, 12])
     assert np.abs(out - ref).max() > 1e-3
+
+
+# ------------------------------------------------------------------------------------------------
+# query-agnostic eviction (Sec. 3.2): anchor = mean of the cached keys, keep the least similar keys
+
+def _keydiff_once(K, V, budget, w, n_first=None):
+    """One block of all keys into an empty cache of `budget` entries (a single eviction round)."""
+    n, hkv, d = K.shape
+    orc = KVCOracle(1, hkv, hkv, d, budget, w, policy="keydiff")
+    q = np.zeros((n, hkv, d))
+    res = orc.prefill_chunk(0, q, K, V, 0)
+    return orc, res
+
+
+def test_keydiff_score_is_one_minus_library_cosine():
+    rng = np.random.default_rng(31)
+    n, d, B, w = 40, 16, 12, 4
+    K = rng.normal(size=(n, 1, d)) + 0.7          # a non-zero mean, so the anchor is well defined
+    V = rng.normal(size=(n, 1, d))
+    orc, res = _keydiff_once(K, V, B, w)
+    mu = torch.from_numpy(K[:, 0]).mean(dim=0, keepdim=True)
+    cos = torch.nn.functional.cosine_similarity(torch.from_numpy(K[: n - w, 0]), mu, dim=1).numpy()
+    assert np.allclose(res.score[0], 1.0 - cos, atol=1e-12)
+    keep = np.sort(np.concatenate([np.argsort(cos, kind="stable")[: B - w], np.arange(n - w, n)]))
+    assert np.array_equal(res.retained_pos[0], keep)
+
+
+def test_keydiff_keeps_the_outlier_and_breaks_ties_by_age():
+    d, n, B, w = 8, 20, 6, 2
+    base = np.ones((1, 1, d))
+    K = np.repeat(base, n, axis=0)
+    K[7, 0] = -np.arange(1, d + 1)                # the one key that points away from everybody else
+    V = np.zeros((n, 1, d))
+    orc, res = _keydiff_once(K, V, B, w)
+    kept = res.retained_pos[0].tolist()
+    assert 7 in kept                               # lowest similarity to the mean: retained
+    # the identical keys tie: the older ones stay, then the protected tail
+    assert kept == [0, 1, 2, 7, n - 2, n - 1]
+
+
+def test_keydiff_invariant_under_common_scaling_and_rotation():
+    rng = np.random.default_rng(32)
+    n, d, B, w = 50, 12, 20, 5
+    K = rng.normal(size=(n, 2, d)) + 0.3
+    V = rng.normal(size=(n, 2, d))
+    _, a = _keydiff_once(K, V, B, w)
+    _, b = _keydiff_once(3.7 * K, V, B, w)
+    R, _ = np.linalg.qr(rng.normal(size=(d, d)))
+    _, c = _keydiff_once(K @ R, V, B, w)
+    for g in range(2):
+        assert np.allclose(a.score[g], b.score[g], atol=1e-12) and np.allclose(a.score[g], c.score[g], atol=1e-12)
+        assert np.array_equal(a.retained_pos[g], b.retained_pos[g]) and np.array_equal(a.retained_pos[g], c.retained_pos[g])
+
+
+def test_keydiff_brute_force_and_budget_invariant():
+    rng = np.random.default_rng(33)
+    n, d, B, w = 11, 6, 7, 2
+    K = rng.normal(size=(n, 1, d)) + 0.5
+    V = rng.normal(size=(n, 1, d))
+    orc, res = _keydiff_once(K, V, B, w)
+    mu = K[:, 0].mean(axis=0)
+    sim = [float(K[j, 0] @ mu / (np.linalg.norm(K[j, 0]) * np.linalg.norm(mu))) for j in range(n - w)]
+    best = min(itertools.combinations(range(n - w), B - w), key=lambda sset: sum(sim[j] for j in sset))
+    assert sorted(best) + [n - 2, n - 1] == res.retained_pos[0].tolist()   # minimal total similarity, unique without ties
+    assert orc.cache_len(0, 0) == B
+    # a zero key has cosine 0 by definition and never produces a NaN
+    K2 = K.copy(); K2[3, 0] = 0.0
+    _, r2 = _keydiff_once(K2, V, B, w)
+    assert np.isfinite(r2.score[0]).all() and r2.score[0][3] == 1.0

@@ -243,10 +243,11 @@ def reference_arm(args, cfg, rank):
 # our arm
 
 class Runner:
-    def __init__(self, cfg, device_index, n_layers=None, flags=0):
+    def __init__(self, cfg, device_index, n_layers=None, flags=0, policy=0):
         from paper_2604_16734_b200.binding import Kvc
         self.cfg = cfg
         self.flags = flags
+        self.policy = policy
         self.L = cfg.n_layers if n_layers is None else n_layers
         self.dev = torch.device("cuda", device_index)
         wl = Workload(cfg, device=self.dev)
@@ -260,7 +261,7 @@ class Runner:
         del wl
         self.O = torch.empty_like(self.Q)
         self.kvc = Kvc(self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk,
-                       cfg.obs_window, device=device_index, flags=flags)
+                       cfg.obs_window, device=device_index, flags=flags, policy=policy)
         self.sched = cfg.chunks()
         # raw pointers of every (block, layer) slice, so the per-call host work is one ctypes call
         self.ptrs = {}
@@ -351,7 +352,7 @@ def profile_pass(r: Runner, steps: int, batched: bool = False):
             kv._check(kv._lib.kvc_prefill_chunk(kv._h, l, q, k, v, n, p, kv.cache[l].data_ptr(), kv.workspace.data_ptr(),
                                                 o, kv._stream()))
             moves = kv.move_counts(0).tolist() if n_c + n > cfg.budget else None
-            fused = cfg.dtype == "bf16" and not (r.flags & 1) and min(cfg.obs_window, n) * cfg.group <= 128
+            fused = r.policy == 1 or (cfg.dtype == "bf16" and not (r.flags & 1) and min(cfg.obs_window, n) * cfg.group <= 128)
             for s, wv in work_of_call(cfg, n, n_c, moves, fused).items():
                 work[s]["bytes"] += wv["bytes"]; work[s]["flops"] += wv["flops"]
         n_c = min(n_c + n, cfg.budget)
@@ -380,6 +381,8 @@ def main():
     ap.add_argument("--workload", default="C2", choices=sorted(CONFIGS))
     ap.add_argument("--mode", default="graph", choices=["graph", "direct", "batched"])
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (0 = all; not a headline run)")
+    ap.add_argument("--policy", default="attn", choices=["attn", "keydiff"],
+                    help="eviction score: query-aware attention score (Eq. 4) or query-agnostic key similarity (Sec. 3.2)")
     ap.add_argument("--flags", type=int, default=0, help="KVC_FLAG_* bits passed to kvc_create (kernel selection, diagnostics)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -409,7 +412,7 @@ def main():
 
     peaks = load_peaks()
     L = args.layers if args.layers else cfg.n_layers
-    r = Runner(cfg, local_rank, L, args.flags)
+    r = Runner(cfg, local_rank, L, args.flags, 1 if args.policy == "keydiff" else 0)
     kv = r.kvc
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -506,7 +509,7 @@ def main():
                 "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
                            "head_dim": cfg.head_dim, "tokens": cfg.n_tokens, "block": cfg.chunk, "budget": cfg.budget,
-                           "obs_window": cfg.obs_window, "mode": args.mode, "parallelism": f"replicas x{world}",
+                           "obs_window": cfg.obs_window, "policy": args.policy, "mode": args.mode, "parallelism": f"replicas x{world}",
                            "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"},
                 "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
                 "kv_bytes": {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,

@@ -42,7 +42,11 @@ typedef struct kvc_ctx kvc_ctx; /* opaque, host memory, created/destroyed by the
 #define KVC_ETIMEOUT -4  /* a bounded device-side wait ran out (reported by kvc_status)                */
 
 typedef enum { KVC_F32 = 0, KVC_BF16 = 1 } kvc_dtype;
-typedef enum { KVC_SCORE_ATTN = 0 /* query-aware score, Eq. 4 */ } kvc_policy;
+typedef enum {
+  KVC_SCORE_ATTN = 0,    /* query-aware score, Eq. 4 */
+  KVC_SCORE_KEYDIFF = 1  /* query-agnostic score, Sec. 3.2: anchor = mean of the cached keys after the append,
+                            score = 1 - cosine(key, anchor); the least similar keys are kept */
+} kvc_policy;
 
 /* flags */
 #define KVC_FLAG_CUDA_CORES 1u /* bf16 only: run attention/score on the CUDA-core kernels used for

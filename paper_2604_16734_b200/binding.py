@@ -16,7 +16,7 @@ from . import build as _build
 
 KVC_OK, KVC_EINVAL, KVC_ESTATE, KVC_ECUDA, KVC_ETIMEOUT = 0, -1, -2, -3, -4
 KVC_F32, KVC_BF16 = 0, 1
-KVC_SCORE_ATTN = 0
+KVC_SCORE_ATTN, KVC_SCORE_KEYDIFF = 0, 1
 KVC_FLAG_CUDA_CORES = 1
 
 EXPORTS = [
@@ -108,7 +108,7 @@ class Kvc:
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: torch.dtype,
                  budget: int, max_chunk: int, obs_window: int = 0, softmax_scale: float = 0.0,
-                 device: int = 0, flags: int = 0, allocate: bool = True):
+                 device: int = 0, flags: int = 0, allocate: bool = True, policy: int = KVC_SCORE_ATTN):
         if not torch.cuda.is_available():
             raise RuntimeError("kvc needs a CUDA device: there is no CPU implementation of the hot path")
         self._lib = lib()
@@ -116,7 +116,7 @@ class Kvc:
         self.device = torch.device("cuda", device)
         code = {torch.float32: KVC_F32, torch.bfloat16: KVC_BF16}[dtype]
         self.cfg = KvcConfig(n_layers, n_q_heads, n_kv_heads, head_dim, code, budget, max_chunk, obs_window,
-                             KVC_SCORE_ATTN, softmax_scale, device, flags)
+                             policy, softmax_scale, device, flags)
         h = ctypes.c_void_p()
         rc = self._lib.kvc_create(ctypes.byref(self.cfg), ctypes.byref(h))
         if rc != KVC_OK:

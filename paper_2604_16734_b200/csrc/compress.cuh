@@ -2,12 +2,13 @@
 // (Alg. 1, Evict) and hole-fill compaction back to the budget (Alg. 1, "reduce cache to budget M").
 //
 // One thread-block cluster of Cn CTAs per (kv-head, layer).
-//   phase 1 (SCORE = true, bf16)  the 128-key tiles of the candidates are dealt round-robin to the CTAs
+//   phase 1 (MODE = kScoreAttention, bf16)  the 128-key tiles of the candidates are dealt round-robin to the CTAs
 //            of the cluster.  Per tile: K tile by TMA, S^T = K_tile Q_obs^T on the tensor cores (keys on
 //            the TMEM lanes, observer rows on the columns), each thread sums 2^(s*scale - lse2) over
 //            the observer columns of its key and writes the score.  Two tiles are in flight per CTA
 //            (two K buffers, two TMEM accumulators, two epilogue warp groups).
-//            With SCORE = false the scores are already in the workspace (CUDA-core score kernel).
+//            MODE = kScoresGiven: the scores are already in the workspace (score kernel of its own).
+//            MODE = kScoreKeyDiff: query-agnostic score 1 - cos(k_j, mean key) (Sec. 3.2), any dtype.
 //   phase 2  cluster barrier; then EVERY CTA reads all scores of its kv-head (L2-resident), builds the
 //            64-bit keys in shared memory and runs the same exact selection redundantly -- cheaper than
 //            a distributed histogram, since the SM-to-SM path is narrow and the other SMs would idle.
@@ -32,6 +33,7 @@ static constexpr int kSelBins = 1 << kDigitBits;
 static constexpr int kMaxKeysSmem = 6144;     // candidates whose keys fit the shared-memory table (48 KB)
 static constexpr int kMaxMovesSmem = 2048;    // moves whose (src, dst) fit the shared-memory tables (16 KB)
 static constexpr int kMaxObsRowsFused = 128;  // observer rows (w * G) the fused scoring phase takes
+static constexpr int kScoresGiven = 0, kScoreAttention = 1, kScoreKeyDiff = 2;   // what phase 1 of compress_kernel does
 static constexpr int kSubTileBytesC = 128 * 128;
 
 __device__ __forceinline__ unsigned long long select_key(float score, int pos) {
@@ -88,7 +90,7 @@ struct CompressSmem {
 // grid (Cn, Hkv, nl), cluster (Cn,1,1), block 512.
 // dynamic smem: the larger of the scoring buffers (two K tiles + up to 128 observer rows) and of the key
 // and move tables (64 KB), + 1 KB.
-template <int D, bool SCORE>
+template <int D, int MODE>
 __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __grid_constant__ CUtensorMap tm_k,
                                                                        const __grid_constant__ CUtensorMap tm_qobs,
                                                                        char* __restrict__ cache, char* __restrict__ ws,
@@ -115,7 +117,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
   pdl_launch_dependents();                        // the next kernel of the stream may set itself up meanwhile
 
   // ------------------------------------------------------------------------------------ phase 1: scores
-  if constexpr (SCORE) {
+  if constexpr (MODE == kScoreAttention) {
     uint8_t* sK = smem;                              // two K tiles
     uint8_t* sQ = smem + 2 * K_TILE_BYTES;           // observer rows
     const int n_tiles = (p.n_cand + 127) / 128;
@@ -226,6 +228,105 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
       tc_fence_after_sync();
       tmem_dealloc(tmem, 256);
     }
+  } else if constexpr (MODE == kScoreKeyDiff) {
+    // Query-agnostic score (Sec. 3.2): anchor mu = mean of the tot keys the cache holds after the append,
+    // score_j = 1 - cos(k_j, mu) for the candidates (>= 0, so its bit pattern orders like an integer; a
+    // zero key or anchor has cosine 0).  A row is read by lpr lanes of 16 bytes; the CTAs of the cluster
+    // take the 128-row tiles round-robin, add their partial sums through distributed shared memory, and
+    // every CTA scores its own tiles (second read of K: L2).
+    float* s_part = reinterpret_cast<float*>(smem);                 // [16 warps][d] partial sums
+    float* s_sum = s_part + (kCompressThreads / 32) * 128;         // [d] this CTA's sum (read by the cluster)
+    float* s_mu = s_sum + 128;                                      // [d] the anchor, [d] = its norm
+    pdl_wait();
+    const int d = p.d, epl = 16 / elem_bytes;                       // elements per 16-byte piece: 8 (bf16) or 4 (fp32)
+    const int lpr = d / epl, rpw = 32 / lpr;                        // lanes per row, rows per warp and step
+    const int sub = lane / lpr, piece = lane % lpr;
+    const long long row_bytes = static_cast<long long>(d) * elem_bytes;
+    const char* Kg = blob + static_cast<long long>(g) * p.cap * row_bytes + piece * 16;
+    auto load_piece = [&](int row, float* f) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(Kg + row * row_bytes);
+      if (elem_bytes == 2) {
+        const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w4[i] << 16); f[2 * i + 1] = __uint_as_float(w4[i] & 0xffff0000u); }
+      } else {
+        f[0] = __uint_as_float(raw.x); f[1] = __uint_as_float(raw.y); f[2] = __uint_as_float(raw.z); f[3] = __uint_as_float(raw.w);
+#pragma unroll
+        for (int i = 4; i < 8; ++i) f[i] = 0.f;
+      }
+    };
+    const int tiles_all = (p.tot + 127) / 128;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    for (int tile = rank; tile < tiles_all; tile += Cn) {
+      const int r_end = min(p.tot, tile * 128 + 128);
+      for (int row = tile * 128 + warp * rpw + sub; row < r_end; row += (kCompressThreads / 32) * rpw) {
+        float f[8];
+        load_piece(row, f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      }
+    }
+    for (int o = lpr; o < 32; o <<= 1) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+    }
+    if (sub == 0)
+      for (int e = 0; e < epl; ++e) s_part[warp * 128 + piece * epl + e] = acc[e];
+    __syncthreads();
+    if (tid < d) {
+      float t = 0.f;
+      for (int w2 = 0; w2 < kCompressThreads / 32; ++w2) t += s_part[w2 * 128 + tid];
+      s_sum[tid] = t;
+    }
+    __syncthreads();
+    if (Cn > 1) { cluster_arrive(); cluster_wait(); }
+    if (tid < d) {
+      float t = 0.f;
+      if (Cn > 1) {
+        const uint32_t a = smem_u32(&s_sum[tid]);
+        for (int rk = 0; rk < Cn; ++rk) t += dsmem_ld_f32(dsmem_addr(a, rk));
+      } else {
+        t = s_sum[tid];
+      }
+      s_mu[tid] = t / static_cast<float>(p.tot);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      float q2 = 0.f;
+      for (int i = lane; i < d; i += 32) q2 += s_mu[i] * s_mu[i];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) q2 += __shfl_xor_sync(0xffffffffu, q2, o);
+      if (lane == 0) s_mu[d] = sqrtf(q2);
+    }
+    __syncthreads();
+    float mu[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mu[e] = e < epl ? s_mu[piece * epl + e] : 0.f;
+    const float mu_norm = s_mu[d];
+    for (int tile = rank; tile < tiles_all; tile += Cn) {
+      const int r_end = min(p.n_cand, tile * 128 + 128);
+      for (int row0 = tile * 128 + warp * rpw; row0 < r_end; row0 += (kCompressThreads / 32) * rpw) {   // warp-uniform bound
+        const int row = row0 + sub;
+        float dot = 0.f, nrm = 0.f;
+        if (row < r_end) {
+          float f[8];
+          load_piece(row, f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) { dot = fmaf(f[e], mu[e], dot); nrm = fmaf(f[e], f[e], nrm); }
+        }
+        for (int o = 1; o < lpr; o <<= 1) {
+          dot += __shfl_xor_sync(0xffffffffu, dot, o);
+          nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
+        }
+        if (row < r_end && piece == 0) {
+          const float den = sqrtf(nrm) * mu_norm;
+          score[row] = den > 0.f ? 1.f - dot / den : 1.f;
+        }
+      }
+    }
+    __syncthreads();
   } else {
     if (tid == 0) pdl_wait();
     __syncthreads();

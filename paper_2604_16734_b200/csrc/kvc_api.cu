@@ -66,7 +66,7 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVC_EINVAL;
   if (cfg->dtype != KVC_F32 && cfg->dtype != KVC_BF16) return KVC_EINVAL;
   if (cfg->budget < 1 || cfg->max_chunk < 1) return KVC_EINVAL;
-  if (cfg->policy != KVC_SCORE_ATTN) return KVC_EINVAL;
+  if (cfg->policy != KVC_SCORE_ATTN && cfg->policy != KVC_SCORE_KEYDIFF) return KVC_EINVAL;
   if (cfg->obs_window < 0) return KVC_EINVAL;
   if (!(cfg->softmax_scale >= 0.f) || isinf(cfg->softmax_scale)) return KVC_EINVAL;
   const int w = cfg->obs_window == 0 ? 32 : cfg->obs_window;
@@ -356,17 +356,17 @@ static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CU
   return cudaLaunchKernelEx(&lc, kvc::attn_tc_kernel<D>, tq, tk, tv, tkin, tvin, (const __nv_bfloat16*)k,
                             (const __nv_bfloat16*)v, (char*)cache, (__nv_bfloat16*)out, (char*)ws, g, S);
 }
-// a2..a4 fused (compress.cuh).  SCORE = false: the scores are already in the workspace.
-template <int D, bool SCORE>
+// a2..a4 fused (compress.cuh).  MODE: kvc::kScoresGiven / kScoreAttention / kScoreKeyDiff.
+template <int D, int MODE>
 static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
                                    int elem_bytes, bool pdl, cudaStream_t st) {
-  const int score_bytes = SCORE ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * kvc::kMaxObsRowsFused * 128 : 0;
+  const int score_bytes = MODE == kvc::kScoreAttention ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * kvc::kMaxObsRowsFused * 128 : 0;
   const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4;
   const int smem_min = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
   const int smem_solo = 120 * 1024;                      // more than half an SM: one CTA per SM
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::compress_kernel<D, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_solo);
+    cudaError_t e = cudaFuncSetAttribute(kvc::compress_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_solo);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -390,7 +390,7 @@ static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const C
   LaunchAttrs la(Cn, pdl);
   lc.attrs = la.at;
   lc.numAttrs = la.n;
-  return cudaLaunchKernelEx(&lc, kvc::compress_kernel<D, SCORE>, tk, tqo, (char*)cache, (char*)ws, g, Cn, elem_bytes);
+  return cudaLaunchKernelEx(&lc, kvc::compress_kernel<D, MODE>, tk, tqo, (char*)cache, (char*)ws, g, Cn, elem_bytes);
 }
 
 template <int D>
@@ -518,8 +518,9 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (e != cudaSuccess) return check_cuda(c, e, "attention launch setup");
   c->launches++;
   if (evict) {
-    const bool fused_score = c->use_tc && g.w * g.G <= kvc::kMaxObsRowsFused;   // few observer rows: score inside the fused kernel
-    if (!fused_score) {
+    const bool keydiff = cf.policy == KVC_SCORE_KEYDIFF;      // query-agnostic: always scored inside the fused kernel
+    const bool fused_score = !keydiff && c->use_tc && g.w * g.G <= kvc::kMaxObsRowsFused;   // few observer rows: likewise
+    if (!fused_score && !keydiff) {
       // a2 score as a kernel of its own (fp32 on CUDA cores; bf16 with more than 128 observer rows per kv-head)
       ProfScope ps(c, 2, st);
       if (c->use_tc) {
@@ -535,9 +536,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     // (a2 +) a3 select + a4 compact
     {
       ProfScope ps(c, 3, st);
-      if (fused_score) e = D == 128 ? launch_compress<128, true>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st)
-                                    : launch_compress<64, true>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st);
-      else e = launch_compress<64, false>(g, tk, tk, cache, ws, (int)c->elem, pdl, st);
+      if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, tk, tk, cache, ws, (int)c->elem, pdl, st);
+      else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st)
+                                         : launch_compress<64, kvc::kScoreAttention>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st);
+      else e = launch_compress<64, kvc::kScoresGiven>(g, tk, tk, cache, ws, (int)c->elem, pdl, st);
     }
     if (e != cudaSuccess) return check_cuda(c, e, "compress launch");
     c->launches++;

@@ -99,14 +99,15 @@ def compare_chunk(kvc, orc, layer, q, k, v, pos0, kv_heads=None, teacher_forced=
     return stats
 
 
-def make_oracle(cfg, n_layers=None) -> KVCOracle:
+def make_oracle(cfg, n_layers=None, policy="attn") -> KVCOracle:
     return KVCOracle(cfg.n_layers if n_layers is None else n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
-                     cfg.budget, cfg.obs_window)
+                     cfg.budget, cfg.obs_window, policy=policy)
 
 
-def run_workload_parity(kvc, wl_cfg, layer_tensors, layers, kv_heads=None, teacher_forced=False, chunks=None):
+def run_workload_parity(kvc, wl_cfg, layer_tensors, layers, kv_heads=None, teacher_forced=False, chunks=None,
+                        policy="attn"):
     """Free-running (or teacher-forced) parity over a whole chunk schedule for the given layers."""
-    orc = make_oracle(wl_cfg)
+    orc = make_oracle(wl_cfg, policy=policy)
     worst = dict(err_out=0.0, err_lse=0.0, err_score=0.0, adopted=0)
     for pos0, n in (wl_cfg.chunks() if chunks is None else chunks):
         for layer in layers:

@@ -14,10 +14,10 @@ from parity_util import compare_chunk, make_oracle, run_workload_parity
 pytestmark = pytest.mark.gpu
 
 
-def _kvc_for(cfg, flags=0, n_layers=None, max_chunk=None, budget=None):
+def _kvc_for(cfg, flags=0, n_layers=None, max_chunk=None, budget=None, policy=0):
     return Kvc(cfg.n_layers if n_layers is None else n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
                cfg.torch_dtype, cfg.budget if budget is None else budget,
-               cfg.chunk if max_chunk is None else max_chunk, cfg.obs_window, flags=flags)
+               cfg.chunk if max_chunk is None else max_chunk, cfg.obs_window, flags=flags, policy=policy)
 
 
 def _layers(cfg, layers):
@@ -86,6 +86,34 @@ def test_full_size_one_layer(name, kv_heads):
     for g in range(cfg.n_kv_heads):
         kept = pos[g, :ln].tolist()
         assert len(set(kept)) == ln and min(kept) >= 0 and max(kept) == cfg.n_tokens - 1
+
+
+# ------------------------------------------------------------------------------------------------
+# query-agnostic eviction (Sec. 3.2): score = 1 - cosine(key, mean of the cached keys)
+
+@pytest.mark.parametrize("name,units,kv_heads", [("C1", None, None), ("C2", None, None), ("C3", 2, None), ("C4", 14, [1, 6]),
+                                                 ("C5", 44, [2])])
+def test_query_agnostic_policy(name, units, kv_heads):
+    cfg = reduced(CONFIGS[name], n_layers=1, n_units=units)
+    kvc = _kvc_for(cfg, policy=binding.KVC_SCORE_KEYDIFF)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=kv_heads, policy="keydiff")
+    assert worst["err_out"] <= (1e-4 if cfg.dtype == "fp32" else 2e-2)
+    assert kvc.cache_view(0)[3] == min(cfg.n_tokens, cfg.budget)
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv", [(torch.float32, 128, 4, 2), (torch.float32, 64, 2, 2), (torch.bfloat16, 64, 8, 4),
+                                            (torch.bfloat16, 128, 6, 1)])
+def test_query_agnostic_policy_ragged(dtype, d, hq, hkv):
+    torch.manual_seed(17)
+    B, c, w = 150, 170, 8
+    from oracle.kvc_oracle import KVCOracle
+    kvc = Kvc(1, hq, hkv, d, dtype, B, c, w, policy=binding.KVC_SCORE_KEYDIFF)
+    orc = KVCOracle(1, hq, hkv, d, B, w, policy="keydiff")
+    p = 0
+    for n in (130, 1, 19, 170, 33, 8, 129):
+        q = torch.randn(n, hq, d).to(dtype); k = (torch.randn(n, hkv, d) + 0.4).to(dtype); v = torch.randn(n, hkv, d).to(dtype)
+        compare_chunk(kvc, orc, 0, q, k, v, p)
+        p += n
 
 
 # ------------------------------------------------------------------------------------------------

@@ -243,7 +243,7 @@ def reference_arm(args, cfg, rank):
 # our arm
 
 class Runner:
-    def __init__(self, cfg, device_index, n_layers=None, flags=0, policy=0):
+    def __init__(self, cfg, device_index, n_layers=None, flags=0, policy=0, hybrid=False):
         from paper_2604_16734_b200.binding import Kvc
         self.cfg = cfg
         self.flags = flags
@@ -262,7 +262,7 @@ class Runner:
         self.O = torch.empty_like(self.Q)
         self.kvc = Kvc(self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk,
                        cfg.obs_window, device=device_index, flags=flags, policy=policy)
-        self.sched = cfg.chunks()
+        self.sched = cfg.chunks_hybrid() if hybrid else cfg.chunks()
         # raw pointers of every (block, layer) slice, so the per-call host work is one ctypes call
         self.ptrs = {}
         for ci, (p, n) in enumerate(self.sched):
@@ -381,6 +381,8 @@ def main():
     ap.add_argument("--workload", default="C2", choices=sorted(CONFIGS))
     ap.add_argument("--mode", default="graph", choices=["graph", "direct", "batched"])
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (0 = all; not a headline run)")
+    ap.add_argument("--hybrid", action="store_true",
+                    help="hybrid schedule (Sec. 4.3): the first B tokens in one pass, block-wise after that")
     ap.add_argument("--policy", default="attn", choices=["attn", "keydiff"],
                     help="eviction score: query-aware attention score (Eq. 4) or query-agnostic key similarity (Sec. 3.2)")
     ap.add_argument("--flags", type=int, default=0, help="KVC_FLAG_* bits passed to kvc_create (kernel selection, diagnostics)")
@@ -412,7 +414,7 @@ def main():
 
     peaks = load_peaks()
     L = args.layers if args.layers else cfg.n_layers
-    r = Runner(cfg, local_rank, L, args.flags, 1 if args.policy == "keydiff" else 0)
+    r = Runner(cfg, local_rank, L, args.flags, 1 if args.policy == "keydiff" else 0, args.hybrid)
     kv = r.kvc
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -509,7 +511,7 @@ def main():
                 "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
                            "head_dim": cfg.head_dim, "tokens": cfg.n_tokens, "block": cfg.chunk, "budget": cfg.budget,
-                           "obs_window": cfg.obs_window, "policy": args.policy, "mode": args.mode, "parallelism": f"replicas x{world}",
+                           "obs_window": cfg.obs_window, "policy": args.policy, "schedule": "hybrid" if args.hybrid else "block-wise", "mode": args.mode, "parallelism": f"replicas x{world}",
                            "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"},
                 "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
                 "kv_bytes": {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,

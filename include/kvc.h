@@ -109,7 +109,9 @@ int kvc_reset(kvc_ctx* ctx, int layer, int n_layers, void* cache, size_t cache_l
 /* The body of Alg. 1's loop for one block and one layer (steps a0..a4 above; Eq. 1, Eq. 4).
  *   q   DEVICE [n][Hq ][d]  queries of the block (already position-encoded), dtype
  *   k,v DEVICE [n][Hkv][d]  keys / values of the block, dtype
- *   n   1 <= n <= max_chunk; pos0 = absolute position of the block's first token
+ *   n   1 <= n <= max_chunk; pos0 = absolute position of the block's first token.  One exception, the
+ *       hybrid schedule the paper uses by default (Sec. 4.3, "processing the first M tokens in one
+ *       pass"): a layer whose cache is EMPTY accepts up to B tokens in one call (nothing is evicted)
  *   cache      DEVICE this layer's blob (kvc_cache_nbytes per_layer bytes); read and written
  *   workspace  DEVICE scratch (kvc_cache_nbytes workspace bytes); calls sharing a workspace must
  *              be ordered on one stream
@@ -133,7 +135,7 @@ int kvc_prefill_chunk_layers(kvc_ctx* ctx, int layer0, int n_layers, const void*
                              long long out_layer_stride, void* stream);
 
 /* Bytes of the DEVICE staging buffer kvc_prefill_chunk_host needs (room for q, k, v and out of a
- * block of max_chunk tokens). */
+ * block of max(max_chunk, B) tokens). */
 int kvc_staging_nbytes(const kvc_ctx* ctx, size_t* nbytes);
 
 /* kvc_prefill_chunk with HOST q/k/v/out (pinned memory recommended): copies the block's q, k, v

@@ -226,17 +226,18 @@ class Kvc:
         return K, V, pos, view.len
 
     def workspace_view(self, slot: int = 0) -> Tuple[torch.Tensor, torch.Tensor]:
-        """(lse [max_chunk][Hq] fp32, score [Hkv][cap] fp32) of the most recent call, aliasing the workspace."""
+        """(lse [max(max_chunk, B)][Hq] fp32, score [Hkv][cap] fp32) of the most recent call, aliasing the workspace."""
         a, b = ctypes.c_void_p(), ctypes.c_void_p()
         self._check(self._lib.kvc_workspace_view(self._h, self.workspace.data_ptr(), slot, ctypes.byref(a),
                                                  ctypes.byref(b)))
         base = self.workspace.data_ptr()
         cap = (self.cfg.budget + self.cfg.max_chunk + 127) // 128 * 128
         lo = a.value - base
-        lse = self.workspace[lo:lo + self.cfg.max_chunk * self.cfg.n_q_heads * 4].view(torch.float32)
+        rows = max(self.cfg.max_chunk, self.cfg.budget)
+        lse = self.workspace[lo:lo + rows * self.cfg.n_q_heads * 4].view(torch.float32)
         so = b.value - base
         score = self.workspace[so:so + self.cfg.n_kv_heads * cap * 4].view(torch.float32)
-        return lse.view(self.cfg.max_chunk, self.cfg.n_q_heads), score.view(self.cfg.n_kv_heads, cap)
+        return lse.view(rows, self.cfg.n_q_heads), score.view(self.cfg.n_kv_heads, cap)
 
     def move_counts(self, slot: int = 0) -> torch.Tensor:
         """int32 [Hkv]: entries moved per kv-head by the most recent compaction of this slot."""

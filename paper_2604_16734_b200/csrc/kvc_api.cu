@@ -90,7 +90,9 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->pos_off = 2 * kv_bytes;
   c->blob_bytes = align_up(2 * kv_bytes + (size_t)cfg->n_kv_heads * c->cap * 4, 1024);
   size_t o = 0;
-  c->lse_off = o;    o = align_up(o + (size_t)cfg->max_chunk * cfg->n_q_heads * 4, 256);
+  // (lse has room for a first block of up to B tokens: the hybrid schedule of Sec. 4.3 fills an empty cache in one pass)
+  const size_t lse_rows = cfg->max_chunk > cfg->budget ? cfg->max_chunk : cfg->budget;
+  c->lse_off = o;    o = align_up(o + lse_rows * cfg->n_q_heads * 4, 256);
   c->score_off = o;  o = align_up(o + (size_t)cfg->n_kv_heads * c->cap * 4, 256);
   c->msrc_off = o;   o = align_up(o + (size_t)cfg->n_kv_heads * cfg->max_chunk * 4, 256);
   c->mdst_off = o;   o = align_up(o + (size_t)cfg->n_kv_heads * cfg->max_chunk * 4, 256);
@@ -416,7 +418,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (!q || !k || !v || !cache || !ws || !out) return fail(c, KVC_EINVAL, "null pointer argument");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(cache) || !aligned16(ws) || !aligned16(out))
     return fail(c, KVC_EINVAL, "pointers must be 16-byte aligned");
-  if (n < 1 || n > cf.max_chunk) return fail(c, KVC_EINVAL, "n = %d outside [1, max_chunk = %d]", n, cf.max_chunk);
+  // Blocks hold at most max_chunk tokens, except that an EMPTY cache may be filled with up to B tokens in one
+  // pass (hybrid schedule, Sec. 4.3 "processing the first M tokens in one pass"): nothing is evicted then.
+  const int n_limit = (c->len[layer0] == 0 && cf.budget > cf.max_chunk) ? cf.budget : cf.max_chunk;
+  if (n < 1 || n > n_limit) return fail(c, KVC_EINVAL, "n = %d outside [1, %d] (max_chunk = %d; up to B = %d into an empty cache)", n, n_limit, cf.max_chunk, cf.budget);
   if (pos0 < 0 || pos0 + n > 0x7fffffffLL) return fail(c, KVC_EINVAL, "pos0 out of range");
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev != cf.device)
@@ -569,8 +574,9 @@ extern "C" int kvc_prefill_chunk_layers(kvc_ctx* c, int layer0, int n_layers, co
 extern "C" int kvc_staging_nbytes(const kvc_ctx* c, size_t* nbytes) {
   if (!live(c)) return KVC_ESTATE;
   if (!nbytes) return KVC_EINVAL;
-  const size_t qb = (size_t)c->cfg.max_chunk * c->cfg.n_q_heads * c->cfg.head_dim * c->elem;
-  const size_t kb = (size_t)c->cfg.max_chunk * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
+  const size_t rows = c->cfg.max_chunk > c->cfg.budget ? c->cfg.max_chunk : c->cfg.budget;   // room for a bulk first block
+  const size_t qb = rows * c->cfg.n_q_heads * c->cfg.head_dim * c->elem;
+  const size_t kb = rows * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
   *nbytes = 2 * align_up(qb, 256) + 2 * align_up(kb, 256);
   return KVC_OK;
 }
@@ -580,7 +586,9 @@ extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host,
                                       void* stream) {
   if (!live(c)) return KVC_ESTATE;
   if (!q_host || !k_host || !v_host || !out_host || !staging) return fail(c, KVC_EINVAL, "null pointer argument");
-  if (n < 1 || n > c->cfg.max_chunk) return fail(c, KVC_EINVAL, "n = %d outside [1, max_chunk = %d]", n, c->cfg.max_chunk);
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, KVC_EINVAL, "layer %d outside [0, %d)", layer, c->cfg.n_layers);
+  const int n_limit = (c->len[layer] == 0 && c->cfg.budget > c->cfg.max_chunk) ? c->cfg.budget : c->cfg.max_chunk;
+  if (n < 1 || n > n_limit) return fail(c, KVC_EINVAL, "n = %d outside [1, %d]", n, n_limit);
   if (!aligned16(staging)) return fail(c, KVC_EINVAL, "staging must be 16-byte aligned");
   cudaStream_t st = (cudaStream_t)stream;
   const size_t qb = (size_t)n * c->cfg.n_q_heads * c->cfg.head_dim * c->elem;

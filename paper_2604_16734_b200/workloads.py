@@ -89,6 +89,19 @@ class WorkloadConfig:
                 r -= n
         return out
 
+    def chunks_hybrid(self) -> List[Tuple[int, int]]:
+        """Hybrid schedule (the paper's default, Sec. 4.3): the first min(B, n_vision) tokens in one pass,
+        the rest of the vision tokens in blocks of ``chunk``, then the text prompt."""
+        first = min(self.budget, self.n_vision)
+        out = [(0, first)]
+        p = first
+        for end in (self.n_vision, self.n_tokens):
+            while p < end:
+                n = min(self.chunk, end - p)
+                out.append((p, n))
+                p += n
+        return out
+
     def scaled(self, **kw) -> "WorkloadConfig":
         return dataclasses.replace(self, **kw)
 

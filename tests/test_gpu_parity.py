@@ -117,6 +117,26 @@ def test_query_agnostic_policy_ragged(dtype, d, hq, hkv):
 
 
 # ------------------------------------------------------------------------------------------------
+# hybrid schedule (Sec. 4.3): the first B tokens in one pass, block-wise after that
+
+@pytest.mark.parametrize("name,units,kv_heads", [("C1", None, None), ("C3", 3, None), ("C4", 14, [0, 7])])
+def test_hybrid_bulk_first_block(name, units, kv_heads):
+    cfg = reduced(CONFIGS[name], n_layers=1, n_units=units)
+    sched = cfg.chunks_hybrid()
+    assert sched[0] == (0, cfg.budget) and sched[0][1] > cfg.chunk
+    kvc = _kvc_for(cfg)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=kv_heads, chunks=sched)
+    assert worst["err_out"] <= (1e-4 if cfg.dtype == "fp32" else 2e-2)
+    assert kvc.cache_view(0)[3] == cfg.budget
+    # the exception is for an empty cache only
+    q, k, v = _layers(cfg, [0])[0]
+    n = cfg.chunk + 1
+    with pytest.raises(KvcError) as e:
+        kvc.prefill_chunk(0, q[:n].cuda(), k[:n].cuda(), v[:n].cuda(), cfg.n_tokens)
+    assert e.value.code == KVC_EINVAL
+
+
+# ------------------------------------------------------------------------------------------------
 # ragged shapes and degenerate cases
 
 @pytest.mark.parametrize("dtype,d,hq,hkv,flags", [
@@ -231,10 +251,10 @@ def test_host_buffer_entry_point():
 
 def test_argument_errors_enqueue_nothing():
     kvc = Kvc(2, 4, 2, 128, torch.bfloat16, 64, 32)
-    q = torch.randn(33, 4, 128, device="cuda").bfloat16(); k = torch.randn(33, 2, 128, device="cuda").bfloat16()
+    q = torch.randn(65, 4, 128, device="cuda").bfloat16(); k = torch.randn(65, 2, 128, device="cuda").bfloat16()
     before = kvc.launch_count()
     with pytest.raises(KvcError) as e:
-        kvc.prefill_chunk(0, q, k, k, 0)                       # n > max_chunk
+        kvc.prefill_chunk(0, q, k, k, 0)                       # n > max_chunk, and > B even for an empty cache
     assert e.value.code == KVC_EINVAL
     with pytest.raises(KvcError) as e:
         kvc._check(kvc._lib.kvc_prefill_chunk(kvc._h, 5, q.data_ptr(), k.data_ptr(), k.data_ptr(), 8, 0,

@@ -48,3 +48,16 @@ def test_vision_tokens_are_spatially_and_temporally_redundant():
     assert corr(x[:-1], x[1:]) > 0.6                      # consecutive frames (rho = 0.9, noise 0.3)
     text = k[cfg.n_vision:].float()
     assert abs(corr(text[:-1], text[1:])) < 0.1           # text tokens are white
+
+
+def test_hybrid_schedule_covers_the_prefix_once():
+    for cfg in CONFIGS.values():
+        sched = cfg.chunks_hybrid()
+        assert sched[0] == (0, min(cfg.budget, cfg.n_vision))
+        pos = 0
+        for p, n in sched:
+            assert p == pos and 1 <= n and (n <= cfg.chunk or p == 0)
+            pos += n
+        assert pos == cfg.n_tokens
+        # vision and text never share a block
+        assert all(not (p < cfg.n_vision < p + n) for p, n in sched)

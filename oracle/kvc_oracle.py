@@ -27,6 +27,10 @@ design notes of the repository):
     normalised over everything the row attends to;
   * ties at the cut-off keep the older entry (smaller position);
   * scores are recomputed from scratch at every eviction round;
+  * proxy-query variant (Sec. 3.2, "proxy query tokens are extracted from the textual prompt"): a call
+    may carry t trailing proxy tokens.  They attend like any other token of the block (causally, after
+    the block's real tokens) and are the observers of the score, but their keys/values never enter the
+    cache; there is then no protected window: all |C| entries compete and the M best stay.
   * query-agnostic policy (Sec. 3.2, "Query-Agnostic Eviction"): the anchor mu is the mean of the
     raw keys the cache holds right after the block was appended, "similarity" is the cosine, and
     the score of an entry is 1 - cos(k_j, mu) (so "lower similarity" = higher score = retained);
@@ -105,14 +109,17 @@ class KVCOracle:
         self.pos[layer][g], self.K[layer][g], self.V[layer][g] = allpos[idx], allK[idx], allV[idx]
 
     # ------------------------------------------------------------------------------------
-    def prefill_chunk(self, layer: int, q, k, v, pos0: int, kv_heads=None) -> ChunkResult:
+    def prefill_chunk(self, layer: int, q, k, v, pos0: int, kv_heads=None, n_proxy: int = 0) -> ChunkResult:
         """One block of Alg. 1 for one layer.  ``kv_heads`` restricts the work to a subset of kv-heads
-        (they are independent); the other heads' state and outputs are left untouched (zeros)."""
+        (they are independent); the other heads' state and outputs are left untouched (zeros).
+        The last ``n_proxy`` rows of q/k/v are proxy query tokens (observers only, never cached)."""
         q = np.asarray(q, dtype=np.float64)
         k = np.asarray(k, dtype=np.float64)
         v = np.asarray(v, dtype=np.float64)
         n = q.shape[0]
         assert q.shape == (n, self.Hq, self.d) and k.shape == (n, self.Hkv, self.d) and v.shape == k.shape
+        assert 0 <= n_proxy < n
+        n_real = n - n_proxy
         G, M = self.G, self.M
         out = np.zeros((n, self.Hq, self.d))
         lse = np.zeros((n, self.Hq))
@@ -130,7 +137,7 @@ class KVCOracle:
             pos = np.concatenate([self.pos[layer][g], pos0 + np.arange(n, dtype=np.int64)])
             K = np.concatenate([self.K[layer][g], k[:, g, :]], axis=0)
             V = np.concatenate([self.V[layer][g], v[:, g, :]], axis=0)
-            tot = n_c + n
+            tot = n_c + n                                   # keys the block's rows can attend to (proxies included)
 
             # 2. attention (Eq. 1).  Row i sees every older cache entry and block keys t <= i.
             visible = np.ones((n, tot), dtype=bool)
@@ -147,6 +154,10 @@ class KVCOracle:
                 P[hh] = E / l
                 out[:, h, :] = P[hh] @ V
 
+            if n_proxy:
+                # the proxies' keys/values are not part of the cache: drop them again
+                tot = n_c + n_real
+                pos, K, V = pos[:tot], K[:tot], V[:tot]
             self._pre_evict[layer][g] = (pos, K, V)
             # Alg. 1: evict only if |C| > M (strict)
             if tot <= M:
@@ -158,11 +169,14 @@ class KVCOracle:
 
             # 3. score (Eq. 4): observers = last w rows of the block; candidates = all entries but the
             #    observers' own w keys, which are always kept
-            w = min(self.obs_window, n)
-            assert w <= M
-            n_cand = tot - w
+            if n_proxy:
+                w, n_cand = n_proxy, tot                    # observers = the proxies; every entry competes
+            else:
+                w = min(self.obs_window, n)
+                assert w <= M
+                n_cand = tot - w
             if self.policy == "attn":
-                score = P[:, n - w:, :n_cand].sum(axis=(0, 1))
+                score = P[:, n - w:, :n_cand].sum(axis=(0, 1))   # P is over all keys the rows saw: the true normaliser
             else:
                 # query-agnostic (Sec. 3.2): anchor = mean of the cached keys, keep the keys least similar to it
                 mu = K.mean(axis=0)
@@ -172,7 +186,7 @@ class KVCOracle:
 
             # 4. select: keep the (M - w) candidates that come first under
             #    (score descending, position ascending); evict the other tot - M (Alg. 1)
-            n_keep = M - w
+            n_keep = M - w if not n_proxy else M
             order = np.lexsort((pos[:n_cand], -score))      # primary key: -score, secondary: pos
             keep_c = order[:n_keep]
             if 0 < n_keep < n_cand:

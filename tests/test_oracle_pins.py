@@ -343,3 +343,60 @@ def test_keydiff_brute_force_and_budget_invariant():
     K2 = K.copy(); K2[3, 0] = 0.0
     _, r2 = _keydiff_once(K2, V, B, w)
     assert np.isfinite(r2.score[0]).all() and r2.score[0][3] == 1.0
+
+
+# ------------------------------------------------------------------------------------------------
+# proxy query tokens (Sec. 3.2): trailing rows that observe but are never cached
+
+def _proxy_setup(seed=41, n_c_blocks=2):
+    rng = np.random.default_rng(seed)
+    hq, hkv, d, M, w = 4, 2, 8, 12, 3
+    orc_a = KVCOracle(1, hq, hkv, d, M, w)
+    orc_b = KVCOracle(1, hq, hkv, d, M, w)
+    blocks = [(rng.normal(size=(7, hq, d)), rng.normal(size=(7, hkv, d)), rng.normal(size=(7, hkv, d))) for _ in range(n_c_blocks)]
+    proxy = (rng.normal(size=(3, hq, d)), rng.normal(size=(3, hkv, d)), rng.normal(size=(3, hkv, d)))
+    return orc_a, orc_b, blocks, proxy, (hq, hkv, d, M)
+
+
+def test_proxy_rows_do_not_change_real_rows_and_are_never_cached():
+    orc_a, orc_b, blocks, proxy, (hq, hkv, d, M) = _proxy_setup()
+    p = 0
+    for q, k, v in blocks:
+        n = q.shape[0]
+        ra = orc_a.prefill_chunk(0, q, k, v, p)                                   # plain block
+        rb = orc_b.prefill_chunk(0, np.concatenate([q, proxy[0]]), np.concatenate([k, proxy[1]]),
+                                 np.concatenate([v, proxy[2]]), p, n_proxy=3)      # same block + proxies
+        assert np.allclose(ra.out, rb.out[:n], atol=1e-13)                         # proxies come last: real rows cannot see them
+        for g in range(hkv):
+            pos = orc_b.pos[0][g]
+            assert len(pos) <= M and pos.max() < p + n                             # no proxy position ever enters the cache
+            assert len(np.unique(pos)) == len(pos)
+        p += n
+
+
+def test_proxy_scores_are_library_softmax_column_sums_and_selection_is_top_m():
+    rng = np.random.default_rng(42)
+    hq = hkv = 1; d = 8; M = 6
+    orc = KVCOracle(1, hq, hkv, d, M, 2)
+    n, t = 10, 3
+    q = rng.normal(size=(n + t, 1, d)); k = rng.normal(size=(n + t, 1, d)); v = rng.normal(size=(n + t, 1, d))
+    res = orc.prefill_chunk(0, q, k, v, 0, n_proxy=t)
+    S = torch.from_numpy(q[:, 0] @ k[:, 0].T) / math.sqrt(d)
+    mask = torch.tril(torch.ones(n + t, n + t, dtype=torch.bool))
+    P = torch.softmax(S.masked_fill(~mask, float("-inf")), dim=1)
+    out_ref = (P @ torch.from_numpy(v[:, 0])).numpy()
+    assert np.allclose(res.out[:, 0], out_ref, atol=1e-12)                         # proxies attend like ordinary tokens
+    score_ref = P[n:, :n].sum(dim=0).numpy()                                       # over the n real entries only
+    assert np.allclose(res.score[0], score_ref, atol=1e-12)
+    keep = np.sort(np.argsort(-score_ref, kind="stable")[:M])                      # no protected window: the M best of all
+    assert np.array_equal(res.retained_pos[0], keep) and orc.cache_len(0, 0) == M
+    best = max(itertools.combinations(range(n), M), key=lambda sset: sum(score_ref[j] for j in sset))
+    assert sorted(best) == keep.tolist()
+
+
+def test_proxy_block_that_fits_the_budget_evicts_nothing():
+    orc_a, orc_b, blocks, proxy, (hq, hkv, d, M) = _proxy_setup(n_c_blocks=1)
+    q, k, v = blocks[0]
+    res = orc_b.prefill_chunk(0, np.concatenate([q, proxy[0]]), np.concatenate([k, proxy[1]]),
+                              np.concatenate([v, proxy[2]]), 0, n_proxy=3)
+    assert not res.evicted and orc_b.cache_len(0, 0) == 7                          # 7 real entries <= M = 12

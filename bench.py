@@ -82,14 +82,14 @@ def ncu_traffic(workload, kernel):
 # ------------------------------------------------------------------------------------------------
 # algorithmic work of one launch (what the method itself has to move / compute)
 
-def work_of_call(cfg, n, n_c, moves_per_head=None, fused_score=True):
-    """Bytes and FLOPs per step kind for ONE layer of one kvc_prefill_chunk call."""
+def work_of_call(cfg, n, n_c, moves_per_head=None, fused_score=True, n_proxy=0):
+    """Bytes and FLOPs per step kind for ONE layer of one kvc_prefill_chunk call (n includes the proxies)."""
     Hq, Hkv, d, sz, B = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.elem_bytes, cfg.budget
-    tot = n_c + n
-    w = min(cfg.obs_window, n)
+    tot = n_c + n - n_proxy
+    w = n_proxy if n_proxy else min(cfg.obs_window, n)
     out = {}
     out["append"] = dict(bytes=2 * 2 * n * d * sz * Hkv + 4 * n * Hkv, flops=0)
-    out["attention"] = dict(bytes=2 * tot * d * sz * Hkv + 2 * n * d * sz * Hq + 4 * Hq * n,
+    out["attention"] = dict(bytes=2 * (n_c + n) * d * sz * Hkv + 2 * n * d * sz * Hq + 4 * Hq * n,
                             flops=4 * Hq * d * (n * n_c + n * (n + 1) // 2))
     if tot > B:
         m = min(n, tot - B) * Hkv if moves_per_head is None else int(sum(moves_per_head))
@@ -243,7 +243,7 @@ def reference_arm(args, cfg, rank):
 # our arm
 
 class Runner:
-    def __init__(self, cfg, device_index, n_layers=None, flags=0, policy=0, hybrid=False):
+    def __init__(self, cfg, device_index, n_layers=None, flags=0, policy=0, hybrid=False, proxy=0):
         from paper_2604_16734_b200.binding import Kvc
         self.cfg = cfg
         self.flags = flags
@@ -259,16 +259,35 @@ class Runner:
             q, k, v = wl.layer(l)
             self.Q[l], self.K[l], self.V[l] = q, k, v
         del wl
-        self.O = torch.empty_like(self.Q)
-        self.kvc = Kvc(self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk,
-                       cfg.obs_window, device=device_index, flags=flags, policy=policy)
         self.sched = cfg.chunks_hybrid() if hybrid else cfg.chunks()
+        # calls: (row offset in the buffers, rows of the call, proxy rows among them, position of the first token)
+        self.calls = [(p, n, 0, p) for p, n in self.sched]
+        self.proxy = proxy
+        if proxy:
+            # proxy query tokens (Sec. 3.2): the first `proxy` text tokens follow every vision block in the input
+            # buffers, so that a call's rows stay contiguous; the text prompt is an ordinary block at the end
+            nv = cfg.n_vision
+            assert 0 < proxy <= cfg.n_text
+            idx, calls, off = [], [], 0
+            for p, n in self.sched:
+                t = proxy if p < nv else 0
+                idx.append(torch.arange(p, p + n, device=self.dev))
+                if t:
+                    idx.append(torch.arange(nv, nv + t, device=self.dev))
+                calls.append((off, n + t, t, p))
+                off += n + t
+            idx = torch.cat(idx)
+            self.Q, self.K, self.V = (x[:, idx].contiguous() for x in (self.Q, self.K, self.V))
+            self.calls = calls
+        self.O = torch.empty_like(self.Q)
+        self.kvc = Kvc(self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk + proxy,
+                       cfg.obs_window, device=device_index, flags=flags, policy=policy)
         # raw pointers of every (block, layer) slice, so the per-call host work is one ctypes call
         self.ptrs = {}
-        for ci, (p, n) in enumerate(self.sched):
+        for ci, (o, n, t, p) in enumerate(self.calls):
             for l in range(self.L):
-                self.ptrs[ci, l] = (self.Q[l, p:p + n].data_ptr(), self.K[l, p:p + n].data_ptr(),
-                                    self.V[l, p:p + n].data_ptr(), self.O[l, p:p + n].data_ptr())
+                self.ptrs[ci, l] = (self.Q[l, o:o + n].data_ptr(), self.K[l, o:o + n].data_ptr(),
+                                    self.V[l, o:o + n].data_ptr(), self.O[l, o:o + n].data_ptr())
         self.graph = None
 
     def step_direct(self):
@@ -277,10 +296,13 @@ class Runner:
         kv.reset()
         ws = kv.workspace.data_ptr()
         cache0, blob = kv.cache.data_ptr(), kv.blob_bytes
-        for ci, (p, n) in enumerate(self.sched):
+        for ci, (_, n, t, p) in enumerate(self.calls):
             for l in range(self.L):
                 q, k, v, o = self.ptrs[ci, l]
-                rc = lib.kvc_prefill_chunk(h, l, q, k, v, n, p, cache0 + l * blob, ws, o, st)
+                if t:
+                    rc = lib.kvc_prefill_chunk_proxy(h, l, q, k, v, n, t, p, cache0 + l * blob, ws, o, st)
+                else:
+                    rc = lib.kvc_prefill_chunk(h, l, q, k, v, n, p, cache0 + l * blob, ws, o, st)
                 if rc:
                     kv._check(rc)
 
@@ -346,16 +368,21 @@ def profile_pass(r: Runner, steps: int, batched: bool = False):
     # exact move counts need one pass with a readback after every call
     kv.reset()
     n_c = 0
-    for ci, (p, n) in enumerate(r.sched):
+    for ci, (_, n, t, p) in enumerate(r.calls):
         for l in range(r.L):
             q, k, v, o = r.ptrs[ci, l]
-            kv._check(kv._lib.kvc_prefill_chunk(kv._h, l, q, k, v, n, p, kv.cache[l].data_ptr(), kv.workspace.data_ptr(),
-                                                o, kv._stream()))
-            moves = kv.move_counts(0).tolist() if n_c + n > cfg.budget else None
-            fused = r.policy == 1 or (cfg.dtype == "bf16" and not (r.flags & 1) and min(cfg.obs_window, n) * cfg.group <= 128)
-            for s, wv in work_of_call(cfg, n, n_c, moves, fused).items():
+            if t:
+                kv._check(kv._lib.kvc_prefill_chunk_proxy(kv._h, l, q, k, v, n, t, p, kv.cache[l].data_ptr(),
+                                                          kv.workspace.data_ptr(), o, kv._stream()))
+            else:
+                kv._check(kv._lib.kvc_prefill_chunk(kv._h, l, q, k, v, n, p, kv.cache[l].data_ptr(), kv.workspace.data_ptr(),
+                                                    o, kv._stream()))
+            moves = kv.move_counts(0).tolist() if n_c + n - t > cfg.budget else None
+            w_call = t if t else min(cfg.obs_window, n)
+            fused = r.policy == 1 or (cfg.dtype == "bf16" and not (r.flags & 1) and w_call * cfg.group <= 128)
+            for s, wv in work_of_call(cfg, n, n_c, moves, fused, t).items():
                 work[s]["bytes"] += wv["bytes"]; work[s]["flops"] += wv["flops"]
-        n_c = min(n_c + n, cfg.budget)
+        n_c = min(n_c + n - t, cfg.budget)
     torch.cuda.synchronize()
     kv.profile_enable(True)
     for _ in range(steps):
@@ -381,6 +408,11 @@ def main():
     ap.add_argument("--workload", default="C2", choices=sorted(CONFIGS))
     ap.add_argument("--mode", default="graph", choices=["graph", "direct", "batched"])
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (0 = all; not a headline run)")
+    ap.add_argument("--block", type=int, default=0, help="override the workload's block size b (Sec. 4.3 block-size study)")
+    ap.add_argument("--budget", type=int, default=0, help="override the workload's budget M")
+    ap.add_argument("--proxy", type=int, default=0,
+                    help="proxy query tokens (Sec. 3.2): the first PROXY text tokens ride along with every vision block as "
+                         "observers and are never cached (graph / direct modes only)")
     ap.add_argument("--hybrid", action="store_true",
                     help="hybrid schedule (Sec. 4.3): the first B tokens in one pass, block-wise after that")
     ap.add_argument("--policy", default="attn", choices=["attn", "keydiff"],
@@ -395,6 +427,8 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     cfg = CONFIGS[args.workload]
+    if args.block or args.budget:
+        cfg = cfg.scaled(chunk=args.block or cfg.chunk, budget=args.budget or cfg.budget)
     if args.impl == "reference":
         reference_arm(args, cfg, rank)
         return
@@ -414,7 +448,11 @@ def main():
 
     peaks = load_peaks()
     L = args.layers if args.layers else cfg.n_layers
-    r = Runner(cfg, local_rank, L, args.flags, 1 if args.policy == "keydiff" else 0, args.hybrid)
+    if args.proxy and (args.mode == "batched"):
+        raise SystemExit("--proxy runs in the graph and direct modes only")
+    r = Runner(cfg, local_rank, L, args.flags, 1 if args.policy == "keydiff" else 0, args.hybrid, args.proxy)
+    if args.proxy:
+        args.no_e2e = True                      # the host-buffer entry point has no proxy variant
     kv = r.kvc
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -466,7 +504,7 @@ def main():
     # ---- the same kernels with all layers in one launch (possible only with synthetic inputs): what the
     #      bandwidth-bound steps reach when a launch carries enough bytes to fill the GPU
     per_b = {}
-    if rank == 0 and not args.no_profile and L > 1:
+    if rank == 0 and not args.no_profile and L > 1 and not args.proxy:
         per_b = profile_pass(r, 3, batched=True)
         for s, d in per_b.items():
             sec = d["ms_total_per_step"] / 1e3
@@ -511,7 +549,7 @@ def main():
                 "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
                            "head_dim": cfg.head_dim, "tokens": cfg.n_tokens, "block": cfg.chunk, "budget": cfg.budget,
-                           "obs_window": cfg.obs_window, "policy": args.policy, "schedule": "hybrid" if args.hybrid else "block-wise", "mode": args.mode, "parallelism": f"replicas x{world}",
+                           "obs_window": cfg.obs_window, "policy": args.policy, "schedule": "hybrid" if args.hybrid else "block-wise", "proxy_tokens": args.proxy, "mode": args.mode, "parallelism": f"replicas x{world}",
                            "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"},
                 "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
                 "kv_bytes": {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,

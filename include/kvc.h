@@ -122,6 +122,19 @@ int kvc_reset(kvc_ctx* ctx, int layer, int n_layers, void* cache, size_t cache_l
 int kvc_prefill_chunk(kvc_ctx* ctx, int layer, const void* q, const void* k, const void* v, int n,
                       long long pos0, void* cache, void* workspace, void* out, void* stream);
 
+/* The query-aware policy with the text prompt known up front (Sec. 3.2: "Proxy query tokens are extracted
+ * from the textual prompt and used to compute cross-attention over cached keys"): the last n_proxy of the
+ * n rows of q/k/v are proxy query tokens.  They are processed like the other tokens of the block (they
+ * attend causally to the cache, the block and the proxies before them, and `out` has their rows too),
+ * they are the observers of Eq. 4 -- with the softmax normaliser of everything they attend to -- but
+ * their keys and values do not stay in the cache, and no entry is protected: all n_c + n - n_proxy
+ * entries compete and the B best stay.  1 <= n_proxy < n <= max_chunk; pos0 is the position of the
+ * block's first real token.  Cache rows beyond the new length are scratch.  Otherwise as
+ * kvc_prefill_chunk. */
+int kvc_prefill_chunk_proxy(kvc_ctx* ctx, int layer, const void* q, const void* k, const void* v, int n,
+                            int n_proxy, long long pos0, void* cache, void* workspace, void* out,
+                            void* stream);
+
 /* Same as kvc_prefill_chunk for `n_layers` consecutive layers in one set of launches (the layer
  * index becomes a grid dimension).  Only meaningful when every layer's q/k/v exist up front
  * (synthetic inputs, or layers of independent models); a real decoder stack cannot use it because

@@ -22,7 +22,7 @@ KVC_FLAG_CUDA_CORES = 1
 EXPORTS = [
     "kvc_create", "kvc_destroy", "kvc_cache_nbytes", "kvc_workspace_init", "kvc_reset",
     "kvc_prefill_chunk", "kvc_prefill_chunk_layers", "kvc_staging_nbytes", "kvc_prefill_chunk_host",
-    "kvc_prefill_chunk_static", "kvc_status_static",
+    "kvc_prefill_chunk_static", "kvc_status_static", "kvc_prefill_chunk_proxy",
     "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
     "kvc_profile_read", "kvc_launch_count", "kvc_last_error",
 ]
@@ -57,6 +57,7 @@ def load_library() -> ctypes.CDLL:
     lib.kvc_workspace_init.argtypes = [vp, vp, vp]
     lib.kvc_reset.argtypes = [vp, i, i, vp, sz, vp]
     lib.kvc_prefill_chunk.argtypes = [vp, i, vp, vp, vp, i, ll, vp, vp, vp, vp]
+    lib.kvc_prefill_chunk_proxy.argtypes = [vp, i, vp, vp, vp, i, i, ll, vp, vp, vp, vp]
     lib.kvc_prefill_chunk_layers.argtypes = [vp, i, i, vp, ll, vp, vp, ll, i, ll, vp, sz, vp, vp, ll, vp]
     lib.kvc_staging_nbytes.argtypes = [vp, psz]
     lib.kvc_prefill_chunk_host.argtypes = [vp, i, vp, vp, vp, i, ll, vp, vp, vp, vp, vp]
@@ -171,6 +172,17 @@ class Kvc:
         self._check(self._lib.kvc_prefill_chunk(self._h, layer, _ptr(q), _ptr(k), _ptr(v), n, pos0,
                                                 self.cache[layer].data_ptr(), self.workspace.data_ptr(),
                                                 _ptr(out), self._stream()))
+        return out
+
+    def prefill_chunk_proxy(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, n_proxy: int, pos0: int,
+                            out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """prefill_chunk whose last ``n_proxy`` rows are proxy query tokens: observers that are never cached."""
+        if out is None:
+            out = torch.empty_like(q)
+        assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and out.is_contiguous()
+        self._check(self._lib.kvc_prefill_chunk_proxy(self._h, layer, _ptr(q), _ptr(k), _ptr(v), q.shape[0], n_proxy, pos0,
+                                                      self.cache[layer].data_ptr(), self.workspace.data_ptr(),
+                                                      _ptr(out), self._stream()))
         return out
 
     def prefill_chunk_layers(self, layer0: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, pos0: int,

@@ -412,7 +412,7 @@ static cudaError_t launch_tc_score(const Geom& g, const CUtensorMap& tk, const C
 
 static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_ls, const void* k, const void* v,
                      long long kv_ls, int n, long long pos0, void* cache, size_t cache_ls, void* ws, void* out,
-                     long long out_ls, cudaStream_t st) {
+                     long long out_ls, cudaStream_t st, int n_proxy = 0) {
   const kvc_config& cf = c->cfg;
   if (layer0 < 0 || nl < 1 || layer0 + nl > cf.n_layers) return fail(c, KVC_EINVAL, "layer range [%d, %d) outside [0, %d)", layer0, layer0 + nl, cf.n_layers);
   if (!q || !k || !v || !cache || !ws || !out) return fail(c, KVC_EINVAL, "null pointer argument");
@@ -445,11 +445,16 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
 
   Geom g;
   memset(&g, 0, sizeof(g));
-  g.n = n; g.n_c = n_c; g.tot = n_c + n; g.B = cf.budget;
-  g.w = c->w_cfg < n ? c->w_cfg : n;
+  if (n_proxy < 0 || n_proxy >= n) return fail(c, KVC_EINVAL, "n_proxy = %d outside [0, n = %d)", n_proxy, n);
+  // Proxy query tokens (the last n_proxy rows) are appended and attended like the rest of the block, but
+  // the cache ends before them: rows tot .. tot + n_proxy are left behind as unused space, the proxies
+  // are the observers, and with no protected window every entry competes for the B places.
+  g.n = n; g.n_c = n_c; g.tot = n_c + n - n_proxy; g.B = cf.budget;
+  g.w = n_proxy ? n_proxy : (c->w_cfg < n ? c->w_cfg : n);
   g.G = c->G; g.Hq = cf.n_q_heads; g.Hkv = cf.n_kv_heads; g.d = cf.head_dim; g.cap = c->cap; g.nl = nl;
   g.max_chunk = cf.max_chunk;
-  g.n_cand = g.tot - g.w; g.n_keep = g.B - g.w;
+  g.n_cand = n_proxy ? g.tot : g.tot - g.w;
+  g.n_keep = n_proxy ? g.B : g.B - g.w;
   g.scale_log2 = c->scale * 1.4426950408889634f;
   g.pos0 = pos0;
   g.q_ls = q_ls; g.kv_ls = kv_ls; g.out_ls = out_ls; g.cache_ls = (long long)cache_ls;
@@ -560,6 +565,13 @@ extern "C" int kvc_prefill_chunk(kvc_ctx* c, int layer, const void* q, const voi
                                  long long pos0, void* cache, void* workspace, void* out, void* stream) {
   if (!live(c)) return KVC_ESTATE;
   return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, workspace, out, 0, (cudaStream_t)stream);
+}
+
+extern "C" int kvc_prefill_chunk_proxy(kvc_ctx* c, int layer, const void* q, const void* k, const void* v, int n,
+                                       int n_proxy, long long pos0, void* cache, void* workspace, void* out, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (n_proxy < 1) return fail(c, KVC_EINVAL, "n_proxy = %d: at least one proxy token is needed (use kvc_prefill_chunk otherwise)", n_proxy);
+  return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, workspace, out, 0, (cudaStream_t)stream, n_proxy);
 }
 
 extern "C" int kvc_prefill_chunk_layers(kvc_ctx* c, int layer0, int n_layers, const void* q, long long q_layer_stride,

@@ -17,7 +17,7 @@ def tolerances(dtype):
 
 
 def compare_chunk(kvc, orc, layer, q, k, v, pos0, kv_heads=None, teacher_forced=False, out_gpu=None,
-                  slot=0, run_gpu=True):
+                  slot=0, run_gpu=True, n_proxy=0):
     """Runs one block on both sides (or only the oracle if run_gpu is False and out_gpu is given) and
     asserts parity.  Returns a dict of error statistics."""
     cfg = kvc.cfg
@@ -34,10 +34,12 @@ def compare_chunk(kvc, orc, layer, q, k, v, pos0, kv_heads=None, teacher_forced=
             Vc[g, :L] = torch.from_numpy(orc.V[layer][g]).to(dev).to(kvc.dtype)
             Pc[g, :L] = torch.from_numpy(orc.pos[layer][g]).to(dev).to(torch.int32)
     pos_before = Pc[:, :len_before].cpu().numpy().astype(np.int64)
-    if run_gpu:
+    if run_gpu and n_proxy:
+        out_gpu = kvc.prefill_chunk_proxy(layer, q.to(dev), k.to(dev), v.to(dev), n_proxy, pos0)
+    elif run_gpu:
         out_gpu = kvc.prefill_chunk(layer, q.to(dev), k.to(dev), v.to(dev), pos0)
     res = orc.prefill_chunk(layer, q.double().numpy(), k.double().numpy(), v.double().numpy(), pos0,
-                            kv_heads=kv_heads)
+                            kv_heads=kv_heads, n_proxy=n_proxy)
     torch.cuda.synchronize()
     assert kvc.status() == 0, kvc.last_error()
     atol_out, atol_lse = tolerances(kvc.dtype)
@@ -57,14 +59,14 @@ def compare_chunk(kvc, orc, layer, q, k, v, pos0, kv_heads=None, teacher_forced=
 
     Kc, Vc, Pc, len_after = kvc.cache_view(layer)
     B = cfg.budget
-    assert len_after == min(len_before + n, B)
+    assert len_after == min(len_before + n - n_proxy, B)
     for g in heads:
         assert orc.cache_len(layer, g) == len_after
         pos_gpu = Pc[g, :len_after].cpu().numpy().astype(np.int64)
         assert len(np.unique(pos_gpu)) == len_after, "duplicate positions in the cache"
         if res.evicted:
-            w = min(cfg.obs_window if cfg.obs_window else 32, n)
-            n_cand = len_before + n - w
+            w = 0 if n_proxy else min(cfg.obs_window if cfg.obs_window else 32, n)   # proxies: nothing is protected
+            n_cand = len_before + n - n_proxy - w
             # candidate j of the GPU (physical order before compaction) has position:
             phys_pos = np.concatenate([pos_before[g], pos0 + np.arange(n)])[:n_cand]
             sg = score_gpu[g, :n_cand].double().cpu().numpy()
@@ -84,7 +86,7 @@ def compare_chunk(kvc, orc, layer, q, k, v, pos0, kv_heads=None, teacher_forced=
                 kept_c = [p for p in ret_g.tolist() if p in cand]
                 drop_c = [p for p in cand if p not in set(ret_g.tolist())]
                 assert len(kept_c) == B - w
-                protected = set(range(pos0 + n - w, pos0 + n))
+                protected = set(range(pos0 + n - n_proxy - w, pos0 + n - n_proxy))
                 assert protected <= set(ret_g.tolist())
                 cutoff = min(so[p] for p in (set(ret_o.tolist()) & cand))
                 assert min(so[p] for p in kept_c) >= max(so[p] for p in drop_c) - GAP_RTOL * abs(cutoff)

@@ -137,6 +137,52 @@ def test_hybrid_bulk_first_block(name, units, kv_heads):
 
 
 # ------------------------------------------------------------------------------------------------
+# proxy query tokens (Sec. 3.2): the text prompt's first tokens ride along with every vision block as
+# observers and are never cached; the text prompt itself is an ordinary block at the end
+
+@pytest.mark.parametrize("name,units,kv_heads,t", [("C1", None, None, 8), ("C2", None, None, 32), ("C3", 2, None, 16),
+                                                   ("C4", 13, [2, 3], 32), ("C5", 40, [4], 32)])
+def test_proxy_query_tokens(name, units, kv_heads, t):
+    cfg = reduced(CONFIGS[name], n_layers=1, n_units=units)
+    q, k, v = _layers(cfg, [0])[0]
+    nv = cfg.n_vision
+    qp, kp, vp = q[nv:nv + t], k[nv:nv + t], v[nv:nv + t]          # the proxies: the first t text tokens
+    kvc = _kvc_for(cfg, max_chunk=cfg.chunk + t)
+    orc = make_oracle(cfg)
+    for pos0, n in cfg.chunks():
+        if pos0 < nv:
+            compare_chunk(kvc, orc, 0, torch.cat([q[pos0:pos0 + n], qp]), torch.cat([k[pos0:pos0 + n], kp]),
+                          torch.cat([v[pos0:pos0 + n], vp]), pos0, kv_heads=kv_heads, n_proxy=t)
+        else:
+            compare_chunk(kvc, orc, 0, q[pos0:pos0 + n], k[pos0:pos0 + n], v[pos0:pos0 + n], pos0, kv_heads=kv_heads)
+    ln = kvc.cache_view(0)[3]
+    assert ln == min(cfg.n_tokens, cfg.budget)
+
+
+def test_proxy_argument_errors():
+    kvc = Kvc(1, 4, 2, 128, torch.bfloat16, 64, 48)
+    x = torch.zeros(40, 4, 128, device="cuda", dtype=torch.bfloat16); y = torch.zeros(40, 2, 128, device="cuda", dtype=torch.bfloat16)
+    for bad in (0, 40, -1):
+        with pytest.raises(KvcError) as e:
+            kvc.prefill_chunk_proxy(0, x, y, y, bad, 0)
+        assert e.value.code == KVC_EINVAL
+    assert kvc.launch_count() == 0
+
+
+# ------------------------------------------------------------------------------------------------
+# the block-size study's shape (Sec. 4.3): 28x28 tiles, block sizes that do and do not align with a tile
+
+@pytest.mark.parametrize("block", [256, 784])
+def test_block_size_study_workload(block):
+    cfg = reduced(CONFIGS["T4"], n_layers=1, n_units=4).scaled(chunk=block)     # 3136 vision tokens > B = 2048
+    kvc = _kvc_for(cfg)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=[1])
+    assert worst["err_out"] <= 2e-2
+    logical, physical, full = kvc.kv_bytes(cfg.n_tokens)
+    assert logical == 2 * 4 * 128 * 2 * 2048 and physical >= 2 * 4 * 128 * 2 * (2048 + block)   # the bound grows with the block
+
+
+# ------------------------------------------------------------------------------------------------
 # ragged shapes and degenerate cases
 
 @pytest.mark.parametrize("dtype,d,hq,hkv,flags", [

@@ -12,6 +12,8 @@ def test_chunk_schedules_match_the_configs():
     assert c["C3"] == [576] * 5 + [128]
     assert c["C4"] == [196] * 64 + [128]
     assert c["C5"] == [1024] * 36 + [256]
+    assert c["T4"] == [784] * 10 + [128]
+    assert [n for _, n in CONFIGS["T4"].scaled(chunk=512).chunks()] == [512] * 15 + [160, 128]
     for cfg in CONFIGS.values():
         sched = cfg.chunks()
         assert sched[0][0] == 0 and sum(n for _, n in sched) == cfg.n_tokens

@@ -152,18 +152,21 @@ __global__ void __launch_bounds__(128) attn_cc_kernel(const T* __restrict__ q, c
 
 // ------------------------------------------------------------------------------------------------
 // a2 score on CUDA cores (Eq. 4): score_j = sum over the w observer rows and the G heads of the
-// group of 2^(s_ij*scale_log2 - lse2_i).  Thread t owns candidate key blockIdx.x*128 + t.
-// grid (ceil(n_cand/128), Hkv, nl), block 128, dynamic smem = 128*(D+4)*4 + 32*D*4 + 32*4 bytes.
+// group of 2^(s_ij*scale_log2 - lse2_i).  A CTA owns 32 candidate keys; four threads share a key and
+// split the observer rows between them (the sum over rows is the long serial chain otherwise).
+// grid (ceil(n_cand/32), Hkv, nl), block 128, dynamic smem = 32*(D+4)*4 + 32*D*4 + 32*4 bytes.
+static constexpr int kScoreCcKeys = 32;
+
 template <typename T, int D>
 __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, const char* __restrict__ cache,
                                                        char* __restrict__ ws, Geom p) {
   constexpr int KS = D + 4;
   extern __shared__ __align__(16) float smem_f[];
-  float* sK = smem_f;                 // [128][KS]
-  float* sQ = sK + 128 * KS;          // [32][D]
-  float* sL = sQ + 32 * D;            // [32]
+  float* sK = smem_f;                          // [32][KS]
+  float* sQ = sK + kScoreCcKeys * KS;          // [32][D]
+  float* sL = sQ + 32 * D;                     // [32]
   const int layer = blockIdx.z, g = blockIdx.y;
-  const int key0 = blockIdx.x * 128;
+  const int key0 = blockIdx.x * kScoreCcKeys;
   const char* blob = cache + layer * p.cache_ls;
   const T* Kc = reinterpret_cast<const T*>(blob) + static_cast<long long>(g) * p.cap * D;
   const T* qb = q + layer * p.q_ls;
@@ -171,13 +174,14 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
   const float* lse = reinterpret_cast<const float*>(slot + p.lse_off);
   float* score = reinterpret_cast<float*>(slot + p.score_off) + static_cast<long long>(g) * p.cap;
 
-  for (int i = threadIdx.x; i < 128 * D; i += 128) {
+  for (int i = threadIdx.x; i < kScoreCcKeys * D; i += 128) {
     const int j = i / D, c = i % D, key = key0 + j;
     sK[j * KS + c] = key < p.n_cand ? to_f32<T>(Kc[static_cast<long long>(key) * D + c]) : 0.f;
   }
   const int rows = p.w * p.G;
+  const int kj = threadIdx.x >> 2, part = threadIdx.x & 3;       // key of the CTA, quarter of the observer rows
   float acc = 0.f;
-  const float4* krow = reinterpret_cast<const float4*>(&sK[threadIdx.x * KS]);
+  const float4* krow = reinterpret_cast<const float4*>(&sK[kj * KS]);
   for (int r0 = 0; r0 < rows; r0 += 32) {
     __syncthreads();
     for (int i = threadIdx.x; i < 32 * D; i += 128) {
@@ -200,7 +204,7 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
     }
     __syncthreads();
     const int rmax = min(32, rows - r0);
-    for (int r = 0; r < rmax; ++r) {
+    for (int r = part; r < rmax; r += 4) {
       const float4* qrow = reinterpret_cast<const float4*>(&sQ[r * D]);
       float s = 0.f;
 #pragma unroll 8
@@ -211,8 +215,10 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
       acc += exp2f(s * p.scale_log2 - sL[r]);
     }
   }
-  const int key = key0 + threadIdx.x;
-  if (key < p.n_cand) score[key] = acc;
+  acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+  acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+  const int key = key0 + kj;
+  if (part == 0 && key < p.n_cand) score[key] = acc;
 }
 
 }  // namespace kvc

@@ -285,14 +285,14 @@ static void launch_cc_attn(const Geom& g, const void* q, void* cache, void* out,
 }
 template <typename T, int D>
 static cudaError_t launch_cc_score(const Geom& g, const void* q, void* cache, void* ws, cudaStream_t st) {
-  const int smem = (128 * (D + 4) + 32 * D + 32) * 4;
+  const int smem = (kvc::kScoreCcKeys * (D + 4) + 32 * D + 32) * 4;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kvc::score_cc_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid((g.n_cand + 127) / 128, g.Hkv, g.nl);
+  dim3 grid((g.n_cand + kvc::kScoreCcKeys - 1) / kvc::kScoreCcKeys, g.Hkv, g.nl);
   kvc::score_cc_kernel<T, D><<<grid, 128, smem, st>>>((const T*)q, (const char*)cache, (char*)ws, g);
   return cudaSuccess;
 }
@@ -531,7 +531,8 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     const bool keydiff = cf.policy == KVC_SCORE_KEYDIFF;      // query-agnostic: always scored inside the fused kernel
     const bool fused_score = !keydiff && c->use_tc && g.w * g.G <= kvc::kMaxObsRowsFused;   // few observer rows: likewise
     if (!fused_score && !keydiff) {
-      // a2 score as a kernel of its own (fp32 on CUDA cores; bf16 with more than 128 observer rows per kv-head)
+      // a2 score as a kernel of its own (fp32 on CUDA cores; bf16 with more than 128 observer rows per kv-head:
+      // fusing up to 256 rows was measured and is slower, the stand-alone kernel spreads the key tiles wider)
       ProfScope ps(c, 2, st);
       if (c->use_tc) {
         e = D == 128 ? launch_tc_score<128>(g, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, tk, tqo, ws, tok_per_group, st);

@@ -32,9 +32,11 @@ static constexpr int kStages = 4;                 // K/V ring slots of the atten
 //   warp  11    only gives its registers away (setmaxnreg works on groups of four warps)
 // a0: before their first turn the threads of tile B copy the CTA's share of the block's keys, values and
 // positions into the cache.
-// The two softmax groups take turns (named barriers): while one tile's exponentials occupy the
-// CUDA cores the tensor pipe runs the other tile's MMAs; without the hand-over both tiles fall into
-// lockstep and the two pipes idle alternately.
+// The two softmax groups take turns on the exponentials (named barriers): while one tile's exponentials
+// occupy the CUDA cores the tensor pipe runs the other tile's MMAs; without the hand-over both tiles fall
+// into lockstep and the two pipes idle alternately.  Loading S and finding the maxima is outside the turn.
+// (Measured and dropped: eight softmax warps per row tile, two threads per row -- no faster, the per-tile
+// chain is not bound by the instruction count per thread.)
 // TMEM columns: S_A/P_A [0,128)  S_B/P_B [128,256)  O_A [256,384)  O_B [384,512).
 // The running output is rescaled lazily: a row keeps its reference maximum until the true maximum
 // has grown by more than 2^8, so P stays below 256 and O rarely needs touching.
@@ -269,10 +271,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     if (active) {
       for (int j = 0; j < Tl; ++j) {
         const int kt = t_begin + j;                           // key tile index
-        // Waits that gave up only skip the arithmetic: the turn barriers are passed on every path, once
-        // per key tile, so the other row tile never waits for a turn that is not handed over.
+        // Waits that gave up only skip the arithmetic: the turn barrier is passed on every path, once per key
+        // tile and warp, so the other row tile never waits for a turn that is not handed over.
         if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[t], j & 1, abort_flag));
-        if (turns) named_barrier(2 + t, 256);
+        bool took_turn = false;
         if (ok) do {
         tc_fence_after_sync();
         uint32_t sr[128];
@@ -320,6 +322,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             }
           }
         }
+        // Only the exponentials are taken in turns: loading S and finding the row maxima overlap the other
+        // tile's exponentials.
+        if (turns) { named_barrier(2 + t, 256); took_turn = true; }
         const float neg_m = -m_ref;
         float ps[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -342,6 +347,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         }
         l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
         } while (0);
+        if (turns && !took_turn) named_barrier(2 + t, 256);   // a wait gave up before the turn was taken: take it now
         if (turns && !(t == 1 && j + 1 == Tl)) named_barrier_arrive(3 - t, 256);
       }
       if (ok && Tl > 0) ok = mbar_wait(&sh.pv_done[t], (Tl - 1) & 1, abort_flag);

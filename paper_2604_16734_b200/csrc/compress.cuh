@@ -243,8 +243,8 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     const int sub = lane / lpr, piece = lane % lpr;
     const long long row_bytes = static_cast<long long>(d) * elem_bytes;
     const char* Kg = blob + static_cast<long long>(g) * p.cap * row_bytes + piece * 16;
-    auto load_piece = [&](int row, float* f) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(Kg + row * row_bytes);
+    auto fetch = [&](int row) { return *reinterpret_cast<const uint4*>(Kg + row * row_bytes); };
+    auto widen = [&](const uint4 raw, float* f) {
       if (elem_bytes == 2) {
         const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -259,13 +259,24 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    constexpr int kRowsInFlight = 4;                               // independent loads per lane: the pass is latency-bound otherwise
+    const int rstep = (kCompressThreads / 32) * rpw;               // rows the CTA covers per step
     for (int tile = rank; tile < tiles_all; tile += Cn) {
       const int r_end = min(p.tot, tile * 128 + 128);
-      for (int row = tile * 128 + warp * rpw + sub; row < r_end; row += (kCompressThreads / 32) * rpw) {
-        float f[8];
-        load_piece(row, f);
+      for (int row = tile * 128 + warp * rpw + sub; row < r_end; row += rstep * kRowsInFlight) {
+        uint4 raw[kRowsInFlight];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] += f[e];
+        for (int u = 0; u < kRowsInFlight; ++u)
+          if (row + u * rstep < r_end) raw[u] = fetch(row + u * rstep);
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+          if (row + u * rstep < r_end) {
+            float f[8];
+            widen(raw[u], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += f[e];
+          }
+        }
       }
     }
     for (int o = lpr; o < 32; o <<= 1) {
@@ -307,22 +318,29 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     const float mu_norm = s_mu[d];
     for (int tile = rank; tile < tiles_all; tile += Cn) {
       const int r_end = min(p.n_cand, tile * 128 + 128);
-      for (int row0 = tile * 128 + warp * rpw; row0 < r_end; row0 += (kCompressThreads / 32) * rpw) {   // warp-uniform bound
-        const int row = row0 + sub;
-        float dot = 0.f, nrm = 0.f;
-        if (row < r_end) {
-          float f[8];
-          load_piece(row, f);
+      for (int row0 = tile * 128 + warp * rpw; row0 < r_end; row0 += rstep * kRowsInFlight) {   // warp-uniform bound
+        uint4 raw[kRowsInFlight];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) { dot = fmaf(f[e], mu[e], dot); nrm = fmaf(f[e], f[e], nrm); }
-        }
-        for (int o = 1; o < lpr; o <<= 1) {
-          dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
-        }
-        if (row < r_end && piece == 0) {
-          const float den = sqrtf(nrm) * mu_norm;
-          score[row] = den > 0.f ? 1.f - dot / den : 1.f;
+        for (int u = 0; u < kRowsInFlight; ++u)
+          if (row0 + sub + u * rstep < r_end) raw[u] = fetch(row0 + sub + u * rstep);
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+          const int row = row0 + sub + u * rstep;
+          float dot = 0.f, nrm = 0.f;
+          if (row < r_end) {
+            float f[8];
+            widen(raw[u], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { dot = fmaf(f[e], mu[e], dot); nrm = fmaf(f[e], f[e], nrm); }
+          }
+          for (int o = 1; o < lpr; o <<= 1) {
+            dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
+          }
+          if (row < r_end && piece == 0) {
+            const float den = sqrtf(nrm) * mu_norm;
+            score[row] = den > 0.f ? 1.f - dot / den : 1.f;
+          }
         }
       }
     }

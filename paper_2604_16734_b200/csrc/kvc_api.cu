@@ -377,7 +377,8 @@ static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const C
   const int n_tiles = (g.n_cand + 127) / 128;
   int Cn = (int)(kvc::kNumSMs / ((long long)g.Hkv * g.nl));
   if (Cn > 8) Cn = 8;
-  if (Cn > (n_tiles + 3) / 4) Cn = (n_tiles + 3) / 4;
+  const int tiles_per_cta = MODE == kvc::kScoreKeyDiff ? 2 : 4;   // the CUDA-core score reads every tile twice: spread it wider
+  if (Cn > (n_tiles + tiles_per_cta - 1) / tiles_per_cta) Cn = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
   if (Cn < 1) Cn = 1;
   // Two CTAs share an SM only when there are more CTAs than SMs (then one scores while the other selects);
   // a launch that fits the GPU asks for more than half an SM's shared memory so that every CTA gets an SM

@@ -4,6 +4,7 @@ Library routines used as independent references: torch's fp64 scaled-dot-product
 attention, torch.softmax, torch.topk, itertools.combinations (brute force).
 """
 import itertools
+import os
 import math
 
 import numpy as np
@@ -400,3 +401,22 @@ def test_proxy_block_that_fits_the_budget_evicts_nothing():
     res = orc_b.prefill_chunk(0, np.concatenate([q, proxy[0]]), np.concatenate([k, proxy[1]]),
                               np.concatenate([v, proxy[2]]), 0, n_proxy=3)
     assert not res.evicted and orc_b.cache_len(0, 0) == 7                          # 7 real entries <= M = 12
+
+
+def test_oracle_reproduces_its_stored_trace_on_c1():
+    """Regression fixture (tests/golden/c1_oracle_trace.txt, written by tests/golden/make_golden.py from the
+    oracle alone): the retained sets, a log-sum-exp and the top score of every block of C1."""
+    import importlib.util
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "golden", "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = open(os.path.join(here, "golden", "c1_oracle_trace.txt")).read().splitlines()
+    now = mod.trace_lines()
+    assert len(stored) == len(now) == 11
+    for a, b in zip(stored[1:], now[1:]):
+        fa, fb = a.split(" | "), b.split(" | ")
+        assert fa[:4] == fb[:4]                                   # schedule, eviction flag, retained set
+        assert abs(float(fa[4]) - float(fb[4])) <= 1e-9 * max(1.0, abs(float(fa[4])))
+        if fa[5] != "-":
+            assert abs(float(fa[5]) - float(fb[5])) <= 1e-9 * abs(float(fa[5]))

@@ -281,6 +281,40 @@ def test_layer_batched_call_matches_per_layer_calls():
         assert torch.equal(Pa[:, :la], Pb[:, :lb]) and torch.equal(Ka[:, :la], Kb[:, :lb]) and torch.equal(Va[:, :la], Vb[:, :lb])
 
 
+def test_cuda_graph_replay_matches_direct_calls():
+    # the benchmark replays the per-(block, layer) calls from a CUDA graph; the programmatic dependencies between
+    # the kernels must survive the capture: same outputs and same caches as the directly issued calls
+    cfg = reduced(CONFIGS["C4"], n_layers=2, n_units=13)
+    wl = Workload(cfg)
+    qs, ks, vs = zip(*[wl.layer(l) for l in range(2)])
+    Q = torch.stack(qs).cuda(); K = torch.stack(ks).cuda(); V = torch.stack(vs).cuda()
+    a = _kvc_for(cfg); b = _kvc_for(cfg)
+    out_a = torch.zeros_like(Q); out_b = torch.zeros_like(Q)
+
+    def run(kvc, out):
+        kvc.reset()
+        for pos0, n in cfg.chunks():
+            for l in range(2):
+                kvc.prefill_chunk(l, Q[l, pos0:pos0 + n], K[l, pos0:pos0 + n], V[l, pos0:pos0 + n], pos0, out[l, pos0:pos0 + n])
+
+    run(a, out_a)
+    run(b, out_b)                                    # warm-up outside the capture (function attributes, driver entry point)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run(b, out_b)
+    out_b.zero_()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert a.status() == 0 and b.status() == 0
+    assert torch.equal(out_a, out_b)
+    for l in range(2):
+        Ka, Va, Pa, la = a.cache_view(l); Kb, Vb, Pb, lb = b.cache_view(l)
+        assert la == lb == cfg.budget
+        assert torch.equal(Pa[:, :la], Pb[:, :lb]) and torch.equal(Ka[:, :la], Kb[:, :lb]) and torch.equal(Va[:, :la], Vb[:, :lb])
+
+
 def test_host_buffer_entry_point():
     cfg = reduced(CONFIGS["C2"], n_layers=1)
     q, k, v = Workload(cfg).layer(0)

@@ -57,9 +57,9 @@ def load_peaks():
 # of the CUDA sources at capture time, and the figure is reported as null once they have changed.
 
 NCU_TRAFFIC = {
-    "sources": "c24fe5b5f95ff980",
-    "bytes_per_launch": {("C2", "attention"): 7409664, ("C2", "compress"): 4203264,
-                         ("C5", "attention"): 29439488, ("C5", "compress"): 12477696},
+    "sources": "60207646f9cd4b0d",
+    "bytes_per_launch": {("C2", "attention"): 7357952, ("C2", "compress"): 4202752,
+                         ("C5", "attention"): 29612544, ("C5", "compress"): 12622336},
 }
 
 

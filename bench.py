@@ -57,19 +57,24 @@ def load_peaks():
 # of the CUDA sources at capture time, and the figure is reported as null once they have changed.
 
 NCU_TRAFFIC = {
-    "sources": "60207646f9cd4b0d",
+    "sources": "f873c698c9891c0c",
     "bytes_per_launch": {("C2", "attention"): 7357952, ("C2", "compress"): 4202752,
                          ("C5", "attention"): 29612544, ("C5", "compress"): 12622336},
 }
 
 
 def kernel_sources_hash():
+    """Hash of the CUDA sources with comments and white space removed (a reworded comment is not a new kernel)."""
     import glob
     import hashlib
+    import re
     h = hashlib.sha256()
     for f in sorted(glob.glob(os.path.join(ROOT, "paper_2604_16734_b200", "csrc", "*"))):
-        with open(f, "rb") as fh:
-            h.update(fh.read())
+        with open(f) as fh:
+            text = fh.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update(re.sub(r"\s+", "", text).encode())
     return h.hexdigest()[:16]
 
 
@@ -408,13 +413,13 @@ def main():
     ap.add_argument("--workload", default="C2", choices=sorted(CONFIGS))
     ap.add_argument("--mode", default="graph", choices=["graph", "direct", "batched"])
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (0 = all; not a headline run)")
-    ap.add_argument("--block", type=int, default=0, help="override the workload's block size b (Sec. 4.3 block-size study)")
+    ap.add_argument("--block", type=int, default=0, help="override the workload's block size b (block-size study, Sec. 5 / Table 4)")
     ap.add_argument("--budget", type=int, default=0, help="override the workload's budget M")
     ap.add_argument("--proxy", type=int, default=0,
                     help="proxy query tokens (Sec. 3.2): the first PROXY text tokens ride along with every vision block as "
                          "observers and are never cached (graph / direct modes only)")
     ap.add_argument("--hybrid", action="store_true",
-                    help="hybrid schedule (Sec. 4.3): the first B tokens in one pass, block-wise after that")
+                    help="hybrid schedule (Sec. 5, Budgeting): the first B tokens in one pass, block-wise after that")
     ap.add_argument("--policy", default="attn", choices=["attn", "keydiff"],
                     help="eviction score: query-aware attention score (Eq. 4) or query-agnostic key similarity (Sec. 3.2)")
     ap.add_argument("--flags", type=int, default=0, help="KVC_FLAG_* bits passed to kvc_create (kernel selection, diagnostics)")

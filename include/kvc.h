@@ -110,8 +110,8 @@ int kvc_reset(kvc_ctx* ctx, int layer, int n_layers, void* cache, size_t cache_l
  *   q   DEVICE [n][Hq ][d]  queries of the block (already position-encoded), dtype
  *   k,v DEVICE [n][Hkv][d]  keys / values of the block, dtype
  *   n   1 <= n <= max_chunk; pos0 = absolute position of the block's first token.  One exception, the
- *       hybrid schedule the paper uses by default (Sec. 4.3, "processing the first M tokens in one
- *       pass"): a layer whose cache is EMPTY accepts up to B tokens in one call (nothing is evicted)
+ *       hybrid schedule the paper uses by default (Sec. 5, Budgeting: the first M tokens go through in a
+ *       single forward): a layer whose cache is EMPTY accepts up to B tokens in one call (nothing is evicted)
  *   cache      DEVICE this layer's blob (kvc_cache_nbytes per_layer bytes); read and written
  *   workspace  DEVICE scratch (kvc_cache_nbytes workspace bytes); calls sharing a workspace must
  *              be ordered on one stream
@@ -122,8 +122,8 @@ int kvc_reset(kvc_ctx* ctx, int layer, int n_layers, void* cache, size_t cache_l
 int kvc_prefill_chunk(kvc_ctx* ctx, int layer, const void* q, const void* k, const void* v, int n,
                       long long pos0, void* cache, void* workspace, void* out, void* stream);
 
-/* The query-aware policy with the text prompt known up front (Sec. 3.2: "Proxy query tokens are extracted
- * from the textual prompt and used to compute cross-attention over cached keys"): the last n_proxy of the
+/* The query-aware policy with the text prompt known up front (Sec. 3.2, Query-Aware Eviction: the observers
+ * are proxy query tokens taken from the text prompt and attend over the cached keys): the last n_proxy of the
  * n rows of q/k/v are proxy query tokens.  They are processed like the other tokens of the block (they
  * attend causally to the cache, the block and the proxies before them, and `out` has their rows too),
  * they are the observers of Eq. 4 -- with the softmax normaliser of everything they attend to -- but

@@ -27,7 +27,7 @@ design notes of the repository):
     normalised over everything the row attends to;
   * ties at the cut-off keep the older entry (smaller position);
   * scores are recomputed from scratch at every eviction round;
-  * proxy-query variant (Sec. 3.2, "proxy query tokens are extracted from the textual prompt"): a call
+  * proxy-query variant (Sec. 3.2: the observers are proxy tokens taken from the text prompt): a call
     may carry t trailing proxy tokens.  They attend like any other token of the block (causally, after
     the block's real tokens) and are the observers of the score, but their keys/values never enter the
     cache; there is then no protected window: all |C| entries compete and the M best stay.

@@ -1,5 +1,5 @@
 // a2 + a3 + a4 in one launch: importance scores (Eq. 4), exact selection of the entries to evict
-// (Alg. 1, Evict) and hole-fill compaction back to the budget (Alg. 1, "reduce cache to budget M").
+// (Alg. 1, Evict) and hole-fill compaction back to the budget M (the last step of Alg. 1's loop body).
 //
 // One thread-block cluster of Cn CTAs per (kv-head, layer).
 //   phase 1 (MODE = kScoreAttention, bf16)  the 128-key tiles of the candidates are dealt round-robin to the CTAs

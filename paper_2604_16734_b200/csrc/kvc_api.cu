@@ -90,7 +90,7 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->pos_off = 2 * kv_bytes;
   c->blob_bytes = align_up(2 * kv_bytes + (size_t)cfg->n_kv_heads * c->cap * 4, 1024);
   size_t o = 0;
-  // (lse has room for a first block of up to B tokens: the hybrid schedule of Sec. 4.3 fills an empty cache in one pass)
+  // (lse has room for a first block of up to B tokens: the hybrid schedule of Sec. 5 (Budgeting) fills an empty cache in one pass)
   const size_t lse_rows = cfg->max_chunk > cfg->budget ? cfg->max_chunk : cfg->budget;
   c->lse_off = o;    o = align_up(o + lse_rows * cfg->n_q_heads * 4, 256);
   c->score_off = o;  o = align_up(o + (size_t)cfg->n_kv_heads * c->cap * 4, 256);
@@ -420,7 +420,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(cache) || !aligned16(ws) || !aligned16(out))
     return fail(c, KVC_EINVAL, "pointers must be 16-byte aligned");
   // Blocks hold at most max_chunk tokens, except that an EMPTY cache may be filled with up to B tokens in one
-  // pass (hybrid schedule, Sec. 4.3 "processing the first M tokens in one pass"): nothing is evicted then.
+  // pass (hybrid schedule, Sec. 5, Budgeting: the first M tokens go through in a single forward): nothing is evicted then.
   const int n_limit = (c->len[layer0] == 0 && cf.budget > cf.max_chunk) ? cf.budget : cf.max_chunk;
   if (n < 1 || n > n_limit) return fail(c, KVC_EINVAL, "n = %d outside [1, %d] (max_chunk = %d; up to B = %d into an empty cache)", n, n_limit, cf.max_chunk, cf.budget);
   if (pos0 < 0 || pos0 + n > 0x7fffffffLL) return fail(c, KVC_EINVAL, "pos0 out of range");

@@ -90,7 +90,7 @@ class WorkloadConfig:
         return out
 
     def chunks_hybrid(self) -> List[Tuple[int, int]]:
-        """Hybrid schedule (the paper's default, Sec. 4.3): the first min(B, n_vision) tokens in one pass,
+        """Hybrid schedule (the paper's default, Sec. 5 "Budgeting"): the first min(B, n_vision) tokens in one pass,
         the rest of the vision tokens in blocks of ``chunk``, then the text prompt."""
         first = min(self.budget, self.n_vision)
         out = [(0, first)]
@@ -116,7 +116,7 @@ CONFIGS = {
                          rho=0.9),
     "C5": WorkloadConfig("C5", 4, 32, 32, 8, 128, "bf16", (12, 12), 256, 256, 1024, 4096, "video",
                          rho=0.95, scene_cut=32),
-    # The axis of the paper's block-size study (Sec. 4.3, Table 4: blocks of 256 / 512 / 784 / 1024 at a budget of
+    # The axis of the paper's block-size study (Sec. 5 "Block size and structural alignment", Table 4: blocks of 256 / 512 / 784 / 1024 at a budget of
     # 2048 on roughly 8k vision tokens in 28x28 tiles), with the attention shape of a 7B model with grouped heads:
     # 28 layers, 28 query / 4 kv heads, d = 128; 10 tiles of 784 tokens + 128 text tokens.  The block size and the
     # budget are meant to be overridden (``scaled(chunk=..., budget=...)``, ``bench.py --block / --budget``).

@@ -117,7 +117,7 @@ def test_query_agnostic_policy_ragged(dtype, d, hq, hkv):
 
 
 # ------------------------------------------------------------------------------------------------
-# hybrid schedule (Sec. 4.3): the first B tokens in one pass, block-wise after that
+# hybrid schedule (Sec. 5, Budgeting): the first B tokens in one pass, block-wise after that
 
 @pytest.mark.parametrize("name,units,kv_heads", [("C1", None, None), ("C3", 3, None), ("C4", 14, [0, 7])])
 def test_hybrid_bulk_first_block(name, units, kv_heads):
@@ -170,7 +170,7 @@ def test_proxy_argument_errors():
 
 
 # ------------------------------------------------------------------------------------------------
-# the block-size study's shape (Sec. 4.3): 28x28 tiles, block sizes that do and do not align with a tile
+# the block-size study's shape (Sec. 5, Table 4): 28x28 tiles, block sizes that do and do not align with a tile
 
 @pytest.mark.parametrize("block", [256, 784])
 def test_block_size_study_workload(block):

@@ -168,7 +168,7 @@ int kvc_prefill_chunk_host(kvc_ctx* ctx, int layer, const void* q_host, const vo
  * move lists, status word) lives in a fixed array of KVC_STATIC_WS_BYTES bytes compiled into the
  * library, which every GPU that loads the library holds until the process exits.
  *   - The configuration must need no more than KVC_STATIC_WS_BYTES of single-layer scratch
- *     (lse 4*Hq*max_chunk + scores 4*Hkv*cap + move lists 8*Hkv*max_chunk + ~1.5 KB); otherwise
+ *     (lse 4*Hq*max(max_chunk, B) + scores 4*Hkv*cap + move lists 8*Hkv*max_chunk + ~1.5 KB); otherwise
  *     the call returns KVC_EINVAL and kvc_last_error names both sizes.  Nothing is enqueued then.
  *   - The first call on a device looks up the device address of the array (once per device, with
  *     that device current); make that first call outside any stream capture.

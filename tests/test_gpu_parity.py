@@ -204,6 +204,34 @@ def test_ragged_blocks(dtype, d, hq, hkv, flags):
         p += n
 
 
+@pytest.mark.parametrize("seed", list(range(12)))
+def test_random_small_configurations(seed):
+    # random shapes, budgets, windows, block lengths, policies and proxy counts against the oracle
+    import random
+    from oracle.kvc_oracle import KVCOracle
+    rnd = random.Random(1000 + seed)
+    dtype = rnd.choice([torch.bfloat16, torch.bfloat16, torch.float32])
+    d = rnd.choice([64, 128])
+    hkv = rnd.choice([1, 2, 3])
+    G = rnd.choice([1, 2, 4, 5, 8, 16])
+    hq = hkv * G
+    w = rnd.choice([1, 4, 16, 32])
+    B = rnd.choice([w, w + 1, 96, 200, 333])
+    B = max(B, w)
+    c = rnd.choice([40, 128, 150, 260])
+    policy = rnd.choice(["attn", "attn", "keydiff"])
+    kvc = Kvc(1, hq, hkv, d, dtype, B, c, w, policy=binding.KVC_SCORE_KEYDIFF if policy == "keydiff" else 0)
+    orc = KVCOracle(1, hq, hkv, d, B, w, policy=policy)
+    torch.manual_seed(seed)
+    p = 0
+    for step in range(6):
+        n = rnd.choice([1, 2, c // 3 + 1, c - 1, c])
+        t = rnd.choice([0, 0, min(n - 1, rnd.choice([1, 3, 8]))]) if n > 1 else 0
+        q = torch.randn(n, hq, d).to(dtype); k = (torch.randn(n, hkv, d) + 0.3).to(dtype); v = torch.randn(n, hkv, d).to(dtype)
+        compare_chunk(kvc, orc, 0, q, k, v, p, n_proxy=t)
+        p += n - t
+
+
 def test_first_block_larger_than_budget_and_window_equal_to_budget():
     torch.manual_seed(8)
     hq, hkv, d = 4, 2, 128

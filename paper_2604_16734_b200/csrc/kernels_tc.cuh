@@ -43,7 +43,7 @@ static constexpr int kStages = 4;                 // K/V ring slots of the atten
 //
 // Key split: with cluster size S the CTA of cluster rank s handles key tiles [s*T/S, (s+1)*T/S) of
 // its row-tile pair and ends with a partial (O, m, l).  The partials are exchanged through
-// distributed shared memory: rank s owns rows [s*128/S, (s+1)*128/S) of both tiles, every CTA pushes
+// distributed shared memory: rank s owns rows [s*128/S, (s+1)*128/S) of both tiles, every CTA copies
 // its partial rows (fp32) into the owner's shared memory with remote stores, the cluster
 // synchronises, and each rank combines and writes its rows.  Nothing but the final result goes to HBM.
 // grid (ceil(ceil(n/TOK)/2) * S, Hkv, nl), cluster (S,1,1), block 384,
@@ -54,6 +54,7 @@ struct TcSmemAttn {
   uint64_t q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_half[2][2], pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
+  float stat[2 * 128 * 2];   // key split: (m, l) of the rows this rank owns, [S sources][2 tiles][rows_per][2], S * rows_per = 128
 };
 
 template <int D>
@@ -382,41 +383,60 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       }
     }
     if (S > 1) {
-      // Combine the partials of the cluster.  Rank s owns rows [s*rows_per, (s+1)*rows_per) of both tiles.
-      // Every softmax thread pushes its row of O (fp32: the output tolerance leaves no room for a 16-bit
-      // exchange format) and its (m, l) into the owner's shared memory with remote stores -- stores are
-      // not waited for, remote loads would be; rows it owns itself are stored locally -- the cluster
-      // synchronises, and each rank reduces its rows from its own shared memory:
+      // Combine the partials of the cluster (S is a power of two).  Rank s owns rows [s*rows_per, (s+1)*rows_per)
+      // of both tiles.  Tile by tile, the softmax threads park their rows of O (fp32: the output tolerance
+      // leaves no room for a 16-bit exchange format) in a local staging tile, then copy it row by row into
+      // the owners' shared memory with remote stores -- stores are not waited for, remote loads would be --
+      // so that every warp instruction writes 512 contiguous bytes (one 16-byte store per thread straight
+      // from the TMEM layout, thread = row, scatters 32 rows per instruction and moved 13 B/clk).  The
+      // cluster synchronises, and each rank reduces its rows from its own shared memory:
       //   O = sum_s 2^(m_s - m*) O_s / sum_s 2^(m_s - m*) l_s.
-      // stage: [S sources][2 tiles][rows_per][D] fp32 over the Q tiles and the ring; the 16-byte chunks of
-      // a row are XOR-swizzled with (row & 7) so that neither the writers (lane = row) nor the readers
-      // (lane = row, same chunk) collide on banks.
-      const int rows_per = (128 + S - 1) / S;
-      float* stage = reinterpret_cast<float*>(smem);
-      float* stat = stage + S * 2 * rows_per * D;               // [S][2][rows_per][2]: m (-inf: row saw no key), l
+      // recv: [S sources][2 tiles][rows_per][D] fp32 over the Q tiles and the first half of the ring; staging
+      // [128][D] behind it; the 16-byte chunks of a row are XOR-swizzled with (row & 7) so that neither the
+      // writers (lane = row) nor the readers (lane = row, same chunk) collide on banks.
+      const int rows_per = 128 / S;
+      float* stage = reinterpret_cast<float*>(smem);            // recv
+      float* stg = stage + 2 * 128 * D;
+      float* stat = sh.stat;                                    // [S][2][rows_per][2]: m (-inf: row saw no key), l
       cluster_arrive();                                         // every CTA is done with its Q tiles and ring
       cluster_wait();
       if (active) {
-        const int owner = r / rows_per, lr = r - owner * rows_per;
-        const int slot = ((split * 2 + t) * rows_per + lr);
-        uint32_t row_addr = smem_u32(stage + slot * D), stat_addr = smem_u32(stat + slot * 2);
-        if (owner != split) { row_addr = dsmem_addr(row_addr, owner); stat_addr = dsmem_addr(stat_addr, owner); }
+        const int nthr = has_B ? 256 : 128;                     // softmax threads that take part
         const bool have = ok && Tl > 0;                         // warp-uniform
+        for (int tt = 0; tt < (has_B ? 2 : 1); ++tt) {
+          if (t == tt) {
+            const int owner = r / rows_per, lr = r - owner * rows_per;
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          if (have) {
-            tmem_ld32(tmem_O + c * 32, o);
-            tmem_wait_ld();
-          } else {
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[32];
+              if (have) {
+                tmem_ld32(tmem_O + c * 32, o);
+                tmem_wait_ld();
+              } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = 0u;
+                for (int i = 0; i < 32; ++i) o[i] = 0u;
+              }
+#pragma unroll
+              for (int k = 0; k < 8; ++k)
+                *reinterpret_cast<uint4*>(stg + r * D + (((c * 8 + k) ^ (lr & 7)) << 2)) = make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+            }
+            uint32_t stat_addr = smem_u32(stat + ((split * 2 + tt) * rows_per + lr) * 2);
+            if (owner != split) stat_addr = dsmem_addr(stat_addr, owner);
+            dsmem_st_v2(stat_addr, (have && l > 0.f) ? m_ref : -INFINITY, have ? l : 0.f);
           }
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            dsmem_st_v4_b32(row_addr + (((c * 8 + k) ^ (lr & 7)) << 4), o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+          named_barrier(1, nthr);                               // the staging tile is complete
+          constexpr int CPR = D / 4;                            // 16-byte chunks per row
+#pragma unroll 4
+          for (int idx = threadIdx.x; idx < 128 * CPR; idx += nthr) {
+            const int row = idx / CPR, chunk = idx % CPR;
+            const int owner = row / rows_per, lr = row - owner * rows_per;
+            const uint4 v4 = *reinterpret_cast<const uint4*>(stg + row * D + chunk * 4);
+            uint32_t dst = smem_u32(stage + ((split * 2 + tt) * rows_per + lr) * D + chunk * 4);
+            if (owner != split) dst = dsmem_addr(dst, owner);
+            dsmem_st_v4_b32(dst, v4.x, v4.y, v4.z, v4.w);
+          }
+          named_barrier(1, nthr);                               // the staging tile may be overwritten
         }
-        dsmem_st_v2(stat_addr, (have && l > 0.f) ? m_ref : -INFINITY, have ? l : 0.f);
       }
       cluster_arrive();                                         // all partials have landed; no remote access after this
       cluster_wait();

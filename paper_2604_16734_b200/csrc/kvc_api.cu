@@ -330,6 +330,7 @@ static int attn_key_splits(const Geom& g) {
   int S = (int)(kvc::kNumSMs / base);
   if (S > 8) S = 8;                    // portable cluster size limit
   if (S > T / 3) S = T / 3;            // the exchange costs about as much as two key tiles: keep three per CTA
+  while (S & (S - 1)) S &= S - 1;      // a power of two: the 128 rows of a tile divide evenly among the ranks
   return S < 1 ? 1 : S;
 }
 

@@ -12,6 +12,11 @@ Modes (all run the same kernels through the C ABI):
   graph    the same calls captured once into a CUDA graph and replayed (no host work per step)
   batched  one kvc_prefill_chunk_layers call per block, the layer index in the launch grid
            (possible only because the synthetic q/k/v of all layers exist up front)
+In the direct and graph modes a layer's score / select / compact is enqueued on the library's side stream
+(KVC_FLAG_ASYNC_COMPRESS) and overlaps the next layer's attention, as it would in a decoder stack, where the
+next layer waits for this layer's output and not for its compacted cache; the step ends after kvc_join, when
+all of it has finished.  --sync-compress keeps everything in stream order.  Per-kernel durations are taken
+in stream order, every kernel alone on the GPU.
 With N > 1 every rank runs an independent replica of the request on its own GPU: the path has no
 cross-GPU exchange, so there is no collective inside the timed region (weak scaling).
 """
@@ -287,6 +292,10 @@ class Runner:
         self.O = torch.empty_like(self.Q)
         self.kvc = Kvc(self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk + proxy,
                        cfg.obs_window, device=device_index, flags=flags, policy=policy)
+        # per-kernel timing wants every kernel alone on the GPU: a second context that keeps compress in stream order
+        self.kvc_in_order = self.kvc if not flags & 16 else Kvc(
+            self.L, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.budget, cfg.chunk + proxy,
+            cfg.obs_window, device=device_index, flags=flags & ~16, policy=policy)
         # raw pointers of every (block, layer) slice, so the per-call host work is one ctypes call
         self.ptrs = {}
         for ci, (o, n, t, p) in enumerate(self.calls):
@@ -310,6 +319,8 @@ class Runner:
                     rc = lib.kvc_prefill_chunk(h, l, q, k, v, n, p, cache0 + l * blob, ws, o, st)
                 if rc:
                     kv._check(rc)
+        if self.flags & 16:              # compress kernels on the side stream: the step ends when they have
+            kv.join()
 
     def step_batched(self):
         kv = self.kvc
@@ -368,6 +379,8 @@ def time_steps(fn, steps, barrier):
 def profile_pass(r: Runner, steps: int, batched: bool = False):
     """Per-kernel CUDA-event durations (on the launching stream) and exact algorithmic work: one call per
     (block, layer), or with `batched` one call per block with the layer index in the launch grid."""
+    saved = (r.kvc, r.flags)
+    r.kvc, r.flags = r.kvc_in_order, r.flags & ~16
     kv, cfg = r.kvc, r.cfg
     work = {s: dict(bytes=0, flops=0) for s in STEPS}
     # exact move counts need one pass with a readback after every call
@@ -395,6 +408,7 @@ def profile_pass(r: Runner, steps: int, batched: bool = False):
     torch.cuda.synchronize()
     ms, cnt = kv.profile_read()
     kv.profile_enable(False)
+    r.kvc, r.flags = saved
     per = {}
     for s in STEPS:
         if cnt[s]:
@@ -423,6 +437,9 @@ def main():
     ap.add_argument("--policy", default="attn", choices=["attn", "keydiff"],
                     help="eviction score: query-aware attention score (Eq. 4) or query-agnostic key similarity (Sec. 3.2)")
     ap.add_argument("--flags", type=int, default=0, help="KVC_FLAG_* bits passed to kvc_create (kernel selection, diagnostics)")
+    ap.add_argument("--sync-compress", action="store_true",
+                    help="keep a layer's score / select / compact in stream order behind its attention instead of "
+                         "on the library's side stream (KVC_FLAG_ASYNC_COMPRESS, the default of the graph / direct modes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
@@ -455,6 +472,9 @@ def main():
     L = args.layers if args.layers else cfg.n_layers
     if args.proxy and (args.mode == "batched"):
         raise SystemExit("--proxy runs in the graph and direct modes only")
+    side_stream = (args.mode != "batched" and not args.sync_compress and cfg.dtype == "bf16" and not args.flags & 1)
+    if side_stream:
+        args.flags |= 16
     r = Runner(cfg, local_rank, L, args.flags, 1 if args.policy == "keydiff" else 0, args.hybrid, args.proxy)
     if args.proxy:
         args.no_e2e = True                      # the host-buffer entry point has no proxy variant
@@ -554,7 +574,8 @@ def main():
                 "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
                            "head_dim": cfg.head_dim, "tokens": cfg.n_tokens, "block": cfg.chunk, "budget": cfg.budget,
-                           "obs_window": cfg.obs_window, "policy": args.policy, "schedule": "hybrid" if args.hybrid else "block-wise", "proxy_tokens": args.proxy, "mode": args.mode, "parallelism": f"replicas x{world}",
+                           "obs_window": cfg.obs_window, "policy": args.policy, "schedule": "hybrid" if args.hybrid else "block-wise", "proxy_tokens": args.proxy, "mode": args.mode,
+                           "compress": "side stream, beside the next layer's attention" if args.flags & 16 else "in stream order", "parallelism": f"replicas x{world}",
                            "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"},
                 "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
                 "kv_bytes": {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,

@@ -55,6 +55,19 @@ typedef enum {
 #define KVC_FLAG_NO_PDL 8u     /* launch the kernels in plain stream order instead of letting each start
                                   while its predecessor drains (programmatic dependent launch) */
 
+#define KVC_FLAG_ASYNC_COMPRESS 16u /* bf16 tensor-core path, kvc_prefill_chunk / _proxy only: score, select and
+                                  compact (Alg. 1's eviction step) of a layer are enqueued on a stream the context
+                                  owns, ordered after the layer's attention, so that they run beside whatever the
+                                  caller enqueues next on its own stream (in a decoder stack the next layer needs
+                                  this layer's output, not its compacted cache).  The layer then uses workspace
+                                  slot `layer` (kvc_workspace_view / kvc_move_counts take that slot).  Contract:
+                                  the call's q must stay unchanged, and the layer's cache must not be read by the
+                                  caller, until the next kvc call on that layer, kvc_reset of it, kvc_status or
+                                  kvc_join has been enqueued on the stream that does so; every kvc call orders
+                                  itself after the pending work of the layers it touches.  Inside a stream
+                                  capture, call kvc_join before ending the capture.  All calls of one context must
+                                  come from one host thread. */
+
 typedef struct {
   int n_layers;        /* L >= 1                                                                 */
   int n_q_heads;       /* Hq, multiple of n_kv_heads; consecutive query heads share a kv-head     */
@@ -199,7 +212,12 @@ int kvc_workspace_view(const kvc_ctx* ctx, void* workspace, int slot, float** ls
  * entries the most recent eviction moved per kv-head during compaction. */
 int kvc_move_counts(const kvc_ctx* ctx, void* workspace, int slot, int** counts);
 
-/* Synchronises `stream` and returns the device status word kept in the workspace: KVC_OK, or
+/* Orders `stream` after every compress kernel that KVC_FLAG_ASYNC_COMPRESS left on the context's own stream
+ * (no host wait; a no-op when nothing is pending).  After it, work enqueued on `stream` sees the compacted
+ * caches, and a stream capture that the calls were part of may end. */
+int kvc_join(kvc_ctx* ctx, void* stream);
+
+/* Joins as kvc_join does, synchronises `stream` and returns the device status word kept in the workspace: KVC_OK, or
  * KVC_ETIMEOUT if a bounded wait inside a kernel gave up (the kernel then left early; results of
  * that call are invalid but the context and the device stay usable). */
 int kvc_status(kvc_ctx* ctx, void* workspace, void* stream);

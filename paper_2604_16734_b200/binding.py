@@ -18,12 +18,13 @@ KVC_OK, KVC_EINVAL, KVC_ESTATE, KVC_ECUDA, KVC_ETIMEOUT = 0, -1, -2, -3, -4
 KVC_F32, KVC_BF16 = 0, 1
 KVC_SCORE_ATTN, KVC_SCORE_KEYDIFF = 0, 1
 KVC_FLAG_CUDA_CORES = 1
+KVC_FLAG_ASYNC_COMPRESS = 16
 
 EXPORTS = [
     "kvc_create", "kvc_destroy", "kvc_cache_nbytes", "kvc_workspace_init", "kvc_reset",
     "kvc_prefill_chunk", "kvc_prefill_chunk_layers", "kvc_staging_nbytes", "kvc_prefill_chunk_host",
     "kvc_prefill_chunk_static", "kvc_status_static", "kvc_prefill_chunk_proxy",
-    "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
+    "kvc_join", "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
     "kvc_profile_read", "kvc_launch_count", "kvc_last_error",
 ]
 
@@ -67,6 +68,7 @@ def load_library() -> ctypes.CDLL:
     lib.kvc_workspace_view.argtypes = [vp, vp, i, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.kvc_move_counts.argtypes = [vp, vp, i, ctypes.POINTER(vp)]
     lib.kvc_status.argtypes = [vp, vp, vp]
+    lib.kvc_join.argtypes = [vp, vp]
     lib.kvc_kv_bytes.argtypes = [vp, ll, psz, psz, psz]
     lib.kvc_profile_enable.argtypes = [vp, i]
     lib.kvc_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
@@ -237,6 +239,12 @@ class Kvc:
         pos = blob[2 * kvb:2 * kvb + hkv * cap * 4].view(torch.int32).view(hkv, cap)
         return K, V, pos, view.len
 
+    def slot_of(self, layer: int) -> int:
+        """Workspace slot of a single-layer call: the layer itself while compress runs on the side stream, else 0."""
+        side = (self.cfg.flags & KVC_FLAG_ASYNC_COMPRESS) and self.dtype == torch.bfloat16 \
+            and not (self.cfg.flags & KVC_FLAG_CUDA_CORES)
+        return layer if side else 0
+
     def workspace_view(self, slot: int = 0) -> Tuple[torch.Tensor, torch.Tensor]:
         """(lse [max(max_chunk, B)][Hq] fp32, score [Hkv][cap] fp32) of the most recent call, aliasing the workspace."""
         a, b = ctypes.c_void_p(), ctypes.c_void_p()
@@ -257,6 +265,10 @@ class Kvc:
         self._check(self._lib.kvc_move_counts(self._h, self.workspace.data_ptr(), slot, ctypes.byref(a)))
         off = a.value - self.workspace.data_ptr()
         return self.workspace[off:off + 4 * self.cfg.n_kv_heads].view(torch.int32)
+
+    def join(self) -> None:
+        """Orders the current stream after compress kernels still pending on the context's side stream."""
+        self._check(self._lib.kvc_join(self._h, self._stream()))
 
     def status(self) -> int:
         return self._lib.kvc_status(self._h, self.workspace.data_ptr(), self._stream())

@@ -21,6 +21,7 @@ struct Geom {
   long long cache_ls;              // layer stride of the cache blobs, bytes
   long long v_off, pos_off;        // byte offsets of V and pos inside a blob (K is at 0)
   long long ws_ls;                 // workspace slot stride, bytes (one slot per batched layer)
+  int slot0;                       // workspace slot of the call's first layer (0 unless compress runs on the side stream)
   long long lse_off, score_off, msrc_off, mdst_off, mcount_off;   // byte offsets inside a slot
 };
 
@@ -28,7 +29,7 @@ static constexpr int kNumSMs = 148;          // B200
 static constexpr int kWsHeaderBytes = 256;   // status word lives at byte 0 of the workspace
 
 __device__ __forceinline__ char* ws_slot(char* ws, const Geom& p, int slot) {
-  return ws + kWsHeaderBytes + static_cast<long long>(slot) * p.ws_ls;
+  return ws + kWsHeaderBytes + static_cast<long long>(p.slot0 + slot) * p.ws_ls;
 }
 
 template <typename T> __device__ __forceinline__ float to_f32(T x);

@@ -38,6 +38,11 @@ struct kvc_ctx {
   bool profiling;
   struct Prof { int kind; cudaEvent_t a, b; };
   std::vector<Prof> prof;
+  // KVC_FLAG_ASYNC_COMPRESS: the side stream, per layer an event after its attention and one after its
+  // compress kernel, and whether that compress may still be running (host objects, created on first use)
+  cudaStream_t side;
+  std::vector<cudaEvent_t> ev_attn, ev_comp;
+  std::vector<char> pending;
   char err[512];
 };
 
@@ -104,6 +109,8 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->encode = nullptr;
   c->use_tc = cfg->dtype == KVC_BF16 && !(cfg->flags & KVC_FLAG_CUDA_CORES);
   c->profiling = false;
+  c->side = nullptr;
+  c->pending.assign(cfg->n_layers, 0);
   c->err[0] = 0;
   *out = c;
   return KVC_OK;
@@ -149,8 +156,45 @@ struct ProfScope {
   ~ProfScope() { if (on) cudaEventRecord(b, st); }
 };
 
+// Makes `st` wait for the compress kernels of layers [l0, l1) that still run on the side stream.
+static int wait_pending(kvc_ctx* c, int l0, int l1, cudaStream_t st) {
+  for (int l = l0; l < l1; ++l) {
+    if (!c->pending[l]) continue;
+    cudaError_t e = cudaStreamWaitEvent(st, c->ev_comp[l], 0);
+    if (e != cudaSuccess) return fail(c, KVC_ECUDA, "cudaStreamWaitEvent: %s", cudaGetErrorString(e));
+    c->pending[l] = 0;
+  }
+  return KVC_OK;
+}
+
+static int ensure_side_stream(kvc_ctx* c) {
+  if (c->side) return KVC_OK;
+  cudaError_t e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
+  if (e != cudaSuccess) { c->side = nullptr; return fail(c, KVC_ECUDA, "cudaStreamCreate: %s", cudaGetErrorString(e)); }
+  c->ev_attn.assign(c->cfg.n_layers, nullptr);
+  c->ev_comp.assign(c->cfg.n_layers, nullptr);
+  for (int l = 0; l < c->cfg.n_layers; ++l) {
+    if ((e = cudaEventCreateWithFlags(&c->ev_attn[l], cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&c->ev_comp[l], cudaEventDisableTiming)) != cudaSuccess)
+      return fail(c, KVC_ECUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+  }
+  return KVC_OK;
+}
+
+extern "C" int kvc_join(kvc_ctx* c, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  return wait_pending(c, 0, c->cfg.n_layers, (cudaStream_t)stream);
+}
+
 extern "C" int kvc_destroy(kvc_ctx* c) {
   if (!live(c)) return KVC_ESTATE;
+  if (c->side) {
+    cudaStreamSynchronize(c->side);
+    for (auto ev : c->ev_attn) if (ev) cudaEventDestroy(ev);
+    for (auto ev : c->ev_comp) if (ev) cudaEventDestroy(ev);
+    cudaStreamDestroy(c->side);
+    c->side = nullptr;
+  }
   drop_events(c);
   c->magic = 0;
   delete c;
@@ -192,6 +236,7 @@ extern "C" int kvc_reset(kvc_ctx* c, int layer, int n_layers, void* cache, size_
   if (!cache || !aligned16(cache)) return fail(c, KVC_EINVAL, "cache pointer null or misaligned");
   if (n_layers > 1 && (cache_layer_stride < c->blob_bytes || cache_layer_stride % 16)) return fail(c, KVC_EINVAL, "cache_layer_stride");
   cudaStream_t st = (cudaStream_t)stream;
+  if (int rc = wait_pending(c, layer, layer + n_layers, st)) return rc;
   for (int i = 0; i < n_layers; ++i) {
     int rc = check_cuda(c, cudaMemsetAsync((char*)cache + (size_t)i * cache_layer_stride, 0, c->blob_bytes, st), "cudaMemsetAsync");
     if (rc) return rc;
@@ -241,7 +286,9 @@ extern "C" int kvc_status(kvc_ctx* c, void* workspace, void* stream) {
   if (!live(c)) return KVC_ESTATE;
   if (!workspace) return KVC_EINVAL;
   int word = 0;
-  int rc = check_cuda(c, cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream), "cudaMemcpyAsync");
+  int rc = wait_pending(c, 0, c->cfg.n_layers, (cudaStream_t)stream);
+  if (rc) return rc;
+  rc = check_cuda(c, cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream), "cudaMemcpyAsync");
   if (rc) return rc;
   rc = check_cuda(c, cudaStreamSynchronize((cudaStream_t)stream), "cudaStreamSynchronize");
   if (rc) return rc;
@@ -414,7 +461,7 @@ static cudaError_t launch_tc_score(const Geom& g, const CUtensorMap& tk, const C
 
 static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_ls, const void* k, const void* v,
                      long long kv_ls, int n, long long pos0, void* cache, size_t cache_ls, void* ws, void* out,
-                     long long out_ls, cudaStream_t st, int n_proxy = 0) {
+                     long long out_ls, cudaStream_t st, int n_proxy = 0, bool allow_async = true) {
   const kvc_config& cf = c->cfg;
   if (layer0 < 0 || nl < 1 || layer0 + nl > cf.n_layers) return fail(c, KVC_EINVAL, "layer range [%d, %d) outside [0, %d)", layer0, layer0 + nl, cf.n_layers);
   if (!q || !k || !v || !cache || !ws || !out) return fail(c, KVC_EINVAL, "null pointer argument");
@@ -462,6 +509,11 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   g.q_ls = q_ls; g.kv_ls = kv_ls; g.out_ls = out_ls; g.cache_ls = (long long)cache_ls;
   g.v_off = (long long)c->v_off; g.pos_off = (long long)c->pos_off;
   g.ws_ls = (long long)c->ws_slot_bytes;
+  // KVC_FLAG_ASYNC_COMPRESS: score / select / compact of a layer run on a side stream, beside whatever the caller
+  // enqueues next (the next layer's attention, in a decoder stack, needs this layer's output, not its compacted
+  // cache); the layer then works in its own workspace slot, and the next call that touches the layer waits
+  const bool async_compress = (cf.flags & 16u) && nl == 1 && allow_async && c->use_tc;
+  g.slot0 = async_compress ? layer0 : 0;
   g.lse_off = c->lse_off; g.score_off = c->score_off; g.msrc_off = c->msrc_off; g.mdst_off = c->mdst_off;
   g.mcount_off = c->mcount_off;
   const bool evict = g.tot > g.B;                      // Alg. 1: "if |C| > M"
@@ -498,8 +550,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     }
   }
 
-  const bool pdl = !(cf.flags & 8u);                   // flag 8: plain stream order between the kernels (diagnostic)
+  const bool pdl_main = !(cf.flags & 8u);              // flag 8: plain stream order between the kernels (diagnostic)
+  const bool pdl = pdl_main;
   cudaError_t e = cudaSuccess;
+  if (int rc = wait_pending(c, layer0, layer0 + nl, st)) return rc;    // a compress kernel of an earlier block may still run
   // a0 append (the tensor-core attention kernel appends by itself)
   if (!c->use_tc) {
     ProfScope ps(c, 0, st);
@@ -530,6 +584,13 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (e != cudaSuccess) return check_cuda(c, e, "attention launch setup");
   c->launches++;
   if (evict) {
+    if (async_compress) {
+      if (int rc = ensure_side_stream(c)) return rc;
+      if ((e = cudaEventRecord(c->ev_attn[layer0], st)) != cudaSuccess || (e = cudaStreamWaitEvent(c->side, c->ev_attn[layer0], 0)) != cudaSuccess)
+        return check_cuda(c, e, "side stream fork");
+      st = c->side;                                           // everything below goes to the side stream
+    }
+    const bool pdl = pdl_main && !async_compress;             // an event, not a kernel, precedes the side stream's launches
     const bool keydiff = cf.policy == KVC_SCORE_KEYDIFF;      // query-agnostic: always scored inside the fused kernel
     const bool fused_score = !keydiff && c->use_tc && g.w * g.G <= kvc::kMaxObsRowsFused;   // few observer rows: likewise
     if (!fused_score && !keydiff) {
@@ -556,6 +617,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     }
     if (e != cudaSuccess) return check_cuda(c, e, "compress launch");
     c->launches++;
+    if (async_compress) {
+      if ((e = cudaEventRecord(c->ev_comp[layer0], st)) != cudaSuccess) return check_cuda(c, e, "side stream event");
+      c->pending[layer0] = 1;
+    }
   }
   int rc = check_cuda(c, cudaGetLastError(), "kernel launch");
   if (rc) return rc;
@@ -616,7 +681,7 @@ extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host,
   if ((rc = check_cuda(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st), "H2D q"))) return rc;
   if ((rc = check_cuda(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, st), "H2D k"))) return rc;
   if ((rc = check_cuda(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, st), "H2D v"))) return rc;
-  rc = run_chunk(c, layer, 1, dq, 0, dk, dv, 0, n, pos0, cache, 0, workspace, dout, 0, st);
+  rc = run_chunk(c, layer, 1, dq, 0, dk, dv, 0, n, pos0, cache, 0, workspace, dout, 0, st, 0, false);   // staging is reused: no side stream
   if (rc) return rc;
   return check_cuda(c, cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st), "D2H out");
 }
@@ -659,7 +724,7 @@ extern "C" int kvc_prefill_chunk_static(kvc_ctx* c, int layer, const void* q, co
   // the array keeps the previous call's contents: only the status word has to start at zero
   rc = check_cuda(c, cudaMemsetAsync(ws, 0, kvc::kWsHeaderBytes, (cudaStream_t)stream), "cudaMemsetAsync(static scratch)");
   if (rc) return rc;
-  return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, ws, out, 0, (cudaStream_t)stream);
+  return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, ws, out, 0, (cudaStream_t)stream, 0, false);
 }
 
 extern "C" int kvc_status_static(kvc_ctx* c, void* stream) {

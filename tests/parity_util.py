@@ -17,7 +17,7 @@ def tolerances(dtype):
 
 
 def compare_chunk(kvc, orc, layer, q, k, v, pos0, kv_heads=None, teacher_forced=False, out_gpu=None,
-                  slot=0, run_gpu=True, n_proxy=0):
+                  slot=None, run_gpu=True, n_proxy=0):
     """Runs one block on both sides (or only the oracle if run_gpu is False and out_gpu is given) and
     asserts parity.  Returns a dict of error statistics."""
     cfg = kvc.cfg
@@ -52,6 +52,7 @@ def compare_chunk(kvc, orc, layer, q, k, v, pos0, kv_heads=None, teacher_forced=
     err_el = np.abs(out_np[:, qh] - ref) / np.maximum(1.0, np.abs(ref) / 4.0)
     err_out = err_el.max()
     assert err_out <= atol_out, f"attention output max-abs error {err_out} > {atol_out} (layer {layer}, pos0 {pos0})"
+    slot = kvc.slot_of(layer) if slot is None else slot
     lse_gpu, score_gpu = kvc.workspace_view(slot)
     err_lse = np.abs(lse_gpu[:n].double().cpu().numpy()[:, qh] - res.lse[:, qh]).max()
     assert err_lse <= atol_lse, f"lse error {err_lse}"

@@ -6,7 +6,8 @@ import pytest
 import torch
 
 from paper_2604_16734_b200 import binding
-from paper_2604_16734_b200.binding import Kvc, KvcError, KVC_FLAG_CUDA_CORES, KVC_EINVAL, KVC_ESTATE
+from paper_2604_16734_b200.binding import (Kvc, KvcError, KVC_FLAG_CUDA_CORES, KVC_FLAG_ASYNC_COMPRESS, KVC_EINVAL,
+                                           KVC_ESTATE)
 from paper_2604_16734_b200.workloads import CONFIGS, Workload, reduced
 
 from parity_util import compare_chunk, make_oracle, run_workload_parity
@@ -74,10 +75,11 @@ def test_c5_long_video_blocks():
 # the benchmark's configurations at FULL size (every block of the whole prefix, the launch geometry the
 # benchmark times: one layer per call), checked on the kv-heads the oracle can follow in reasonable time
 
-@pytest.mark.parametrize("name,kv_heads", [("C2", None), ("C3", None), ("C4", [0, 5]), ("C5", [3])])
-def test_full_size_one_layer(name, kv_heads):
+@pytest.mark.parametrize("name,kv_heads,flags", [("C2", None, 0), ("C3", None, 0), ("C4", [0, 5], 0), ("C5", [3], 0),
+                                                 ("C2", None, KVC_FLAG_ASYNC_COMPRESS)])
+def test_full_size_one_layer(name, kv_heads, flags):
     cfg = reduced(CONFIGS[name], n_layers=1)
-    kvc = _kvc_for(cfg)
+    kvc = _kvc_for(cfg, flags)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=kv_heads)
     assert worst["err_out"] <= 2e-2
     # the cache never exceeds the budget, and ends exactly at it once the prefix is longer than B
@@ -307,6 +309,57 @@ def test_layer_batched_call_matches_per_layer_calls():
         Ka, Va, Pa, la = a.cache_view(l); Kb, Vb, Pb, lb = b.cache_view(l)
         assert la == lb == cfg.budget
         assert torch.equal(Pa[:, :la], Pb[:, :lb]) and torch.equal(Ka[:, :la], Kb[:, :lb]) and torch.equal(Va[:, :la], Vb[:, :lb])
+
+
+@pytest.mark.parametrize("name,units,n_layers,graph", [("C2", None, 4, False), ("C2", None, 4, True),
+                                                        ("C4", 13, 3, False), ("C4", 13, 3, True), ("C3", 2, 2, False)])
+def test_compress_on_side_stream_matches_in_order_compress(name, units, n_layers, graph):
+    # with KVC_FLAG_ASYNC_COMPRESS a layer's eviction runs beside the next layer's attention; the kernels and their
+    # inputs are the same, so outputs and caches must equal the in-order run bit for bit, directly and from a graph
+    cfg = reduced(CONFIGS[name], n_layers=n_layers, n_units=units)
+    wl = Workload(cfg)
+    qs, ks, vs = zip(*[wl.layer(l) for l in range(n_layers)])
+    Q = torch.stack(qs).cuda(); K = torch.stack(ks).cuda(); V = torch.stack(vs).cuda()
+    a = _kvc_for(cfg); b = _kvc_for(cfg, KVC_FLAG_ASYNC_COMPRESS)
+    out_a = torch.zeros_like(Q); out_b = torch.zeros_like(Q)
+
+    def run(kvc, out):
+        kvc.reset()
+        for pos0, n in cfg.chunks():
+            for l in range(n_layers):
+                kvc.prefill_chunk(l, Q[l, pos0:pos0 + n], K[l, pos0:pos0 + n], V[l, pos0:pos0 + n], pos0, out[l, pos0:pos0 + n])
+        kvc.join()
+
+    run(a, out_a)
+    run(b, out_b)
+    torch.cuda.synchronize()
+    if graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            run(b, out_b)
+        out_b.zero_()
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+    assert a.status() == 0 and b.status() == 0
+    assert torch.equal(out_a, out_b)
+    for l in range(n_layers):
+        Ka, Va, Pa, la = a.cache_view(l); Kb, Vb, Pb, lb = b.cache_view(l)
+        assert la == lb == min(cfg.budget, cfg.n_tokens)
+        assert torch.equal(Pa[:, :la], Pb[:, :lb]) and torch.equal(Ka[:, :la], Kb[:, :lb]) and torch.equal(Va[:, :la], Vb[:, :lb])
+        # each layer kept its own lse / score slot
+        lse_a, sc_a = a.workspace_view(0) if l == n_layers - 1 else (None, None)
+        lse_b, sc_b = b.workspace_view(b.slot_of(l))
+        if lse_a is not None:
+            n_last = cfg.chunks()[-1][1]
+            assert torch.equal(lse_a[:n_last], lse_b[:n_last])
+
+
+def test_compress_on_side_stream_against_the_oracle_two_layers():
+    cfg = reduced(CONFIGS["C4"], n_layers=2, n_units=9)
+    kvc = _kvc_for(cfg, KVC_FLAG_ASYNC_COMPRESS)
+    worst = run_workload_parity(kvc, cfg, _layers(cfg, [0, 1]), [0, 1], kv_heads=[2, 7])
+    assert worst["err_out"] <= 2e-2
 
 
 def test_cuda_graph_replay_matches_direct_calls():

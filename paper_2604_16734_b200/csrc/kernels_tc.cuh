@@ -167,8 +167,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         const uint32_t q_lo = smem_desc_lo(smem_u32(sQ) + t * TILE_BYTES, 16);          // K-major operand
         const uint32_t k_lo0 = smem_desc_lo(smem_u32(ring), 16);                        // K-major operand
         const uint32_t v_lo0 = smem_desc_lo(smem_u32(ring), kSubTileBytes);             // MN-major operand
-        const uint32_t tS = tmem + t * 128, tO = tmem + 256 + t * 128;
-        auto issue_S = [&](int slot) {             // S_t = Q_t K^T, 16 of the d columns per MMA
+        const uint32_t tO = tmem + 256 + t * 128;
+        // A CTA with one row tile has the other tile's S columns to spare: S alternates between the two buffers, and
+        // S of key tile j+1 is queued before P V of tile j, so that the softmax threads find it waiting.
+        const bool dbuf = !has_B;
+        auto s_cols = [&](int j) { return tmem + (dbuf ? (j & 1) : t) * 128; };
+        auto s_bar = [&](int j) { return &sh.s_full[dbuf ? (j & 1) : t]; };
+        auto issue_S = [&](int slot, uint32_t tS) {  // S_t = Q_t K^T, 16 of the d columns per MMA
           const uint32_t k_lo = k_lo0 + slot * (TILE_BYTES >> 4);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
@@ -176,7 +181,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             mma_ss_lh(tS, q_lo + off, hi, k_lo + off, hi, idesc_qk, kk > 0);
           }
         };
-        auto issue_PV = [&](int slot, int half, bool acc) {   // O_t += P_t V, 16 keys per MMA, 64 keys per half
+        auto issue_PV = [&](int slot, int half, bool acc, uint32_t tS) {   // O_t += P_t V, 16 keys per MMA, 64 keys per half
           const uint32_t v_lo = v_lo0 + slot * (TILE_BYTES >> 4);
 #pragma unroll
           for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
@@ -185,30 +190,39 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         bool ok = mbar_wait(&sh.q_full[t], 0, abort_flag) && mbar_wait(&sh.kv_full[0], 0, abort_flag);
         if (ok) {
           tc_fence_after_sync();
-          issue_S(0);
-          mma_commit(&sh.s_full[t]);
+          issue_S(0, s_cols(0));
+          mma_commit(s_bar(0));
           mma_commit(&sh.kv_empty[0]);
         }
+        if (ok && dbuf && Tl > 1) {                  // K_1 sits in ring slot 2
+          ok = mbar_wait(&sh.kv_full[2], 0, abort_flag);
+          if (ok) {
+            tc_fence_after_sync();
+            issue_S(2, s_cols(1));
+            mma_commit(s_bar(1));
+            mma_commit(&sh.kv_empty[2]);
+          }
+        }
         for (int j = 0; j < Tl && ok; ++j) {
-          const int iv = 2 * j + 1, ik = 2 * j + 2;
+          const int jn = dbuf ? j + 2 : j + 1;       // the key tile whose S is queued behind P V of tile j
+          const int iv = 2 * j + 1, ik = 2 * jn;
           const int slotV = iv % kStages, slotK = ik % kStages;
-          const bool more = j + 1 < Tl;
           ok = mbar_wait(&sh.p_half[t][0], j & 1, abort_flag) && mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          issue_PV(slotV, 0, j > 0);
+          issue_PV(slotV, 0, j > 0, s_cols(j));
           ok = mbar_wait(&sh.p_half[t][1], j & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          issue_PV(slotV, 1, true);
+          issue_PV(slotV, 1, true, s_cols(j));
           mma_commit(&sh.pv_done[t]);
           mma_commit(&sh.kv_empty[slotV]);
-          if (more) {
+          if (jn < Tl) {
             ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
-            issue_S(slotK);
-            mma_commit(&sh.s_full[t]);
+            issue_S(slotK, s_cols(jn));              // overwrites P of tile jn - 2, whose P V is queued ahead of it
+            mma_commit(s_bar(jn));
             mma_commit(&sh.kv_empty[slotK]);
           }
         }
@@ -228,7 +242,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     const int tok = tok0 + r / p.G, hh = r % p.G;
     const bool row_valid = r < rows && tok < p.n;
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t tmem_S = tmem + t * 128 + lane_addr, tmem_O = tmem + 256 + t * 128 + lane_addr;
+    const uint32_t tmem_O = tmem + 256 + t * 128 + lane_addr;
+    const bool dbuf = !has_B;                                // one row tile: S alternates between both tiles' columns
     float m_ref = -INFINITY, l = 0.f;                        // reference maximum (log2 units) and row sum
     bool ok = true;
     const bool active = t == 0 || has_B;
@@ -274,7 +289,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         const int kt = t_begin + j;                           // key tile index
         // Waits that gave up only skip the arithmetic: the turn barrier is passed on every path, once per key
         // tile and warp, so the other row tile never waits for a turn that is not handed over.
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[t], j & 1, abort_flag));
+        const uint32_t tmem_S = tmem + (dbuf ? (j & 1) : t) * 128 + lane_addr;
+        if (ok) ok = __all_sync(0xffffffffu, dbuf ? mbar_wait(&sh.s_full[j & 1], (j >> 1) & 1, abort_flag)
+                                                  : mbar_wait(&sh.s_full[t], j & 1, abort_flag));
         bool took_turn = false;
         if (ok) do {
         tc_fence_after_sync();
@@ -448,38 +465,29 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           const int lr = rem % nrows, cg = rem / nrows, r = r0 + lr;
           const int tok = (t ? tokB : tokA) + r / p.G, hh = r % p.G;
           if (!(r < rows && tok < p.n)) continue;
-          float ms[8], wt[8];
+          // (the loops over the sources are kept rolled: this code runs once per CTA, straight-line copies of it
+          // cost more in instruction fetch than the loop does in branches)
           float m_all = -INFINITY;
-#pragma unroll
-          for (int s = 0; s < 8; ++s) {
-            ms[s] = -INFINITY;
-            if (s < S) ms[s] = stat[((s * 2 + t) * rows_per + lr) * 2];
-            m_all = fmaxf(m_all, ms[s]);
-          }
+#pragma unroll 1
+          for (int s = 0; s < S; ++s) m_all = fmaxf(m_all, stat[((s * 2 + t) * rows_per + lr) * 2]);
           float L = 0.f;
-#pragma unroll
-          for (int s = 0; s < 8; ++s) {
-            wt[s] = 0.f;
-            if (s < S && ms[s] != -INFINITY) {
-              wt[s] = fast_exp2(ms[s] - m_all);
-              L = fmaf(wt[s], stat[((s * 2 + t) * rows_per + lr) * 2 + 1], L);
-            }
-          }
           float acc[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll 1
+          for (int s = 0; s < S; ++s) {
+            const float2 ml = *reinterpret_cast<const float2*>(stat + ((s * 2 + t) * rows_per + lr) * 2);
+            if (ml.x == -INFINITY) continue;                  // this source saw no key of the row
+            const float wt = fast_exp2(ml.x - m_all);
+            L = fmaf(wt, ml.y, L);
+            const float* row = stage + ((s * 2 + t) * rows_per + lr) * D;
 #pragma unroll
-          for (int s = 0; s < 8; ++s) {
-            if (s < S && wt[s] != 0.f) {
-              const float* row = stage + ((s * 2 + t) * rows_per + lr) * D;
-#pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const float4 v4 = *reinterpret_cast<const float4*>(row + (((cg * 8 + k) ^ (lr & 7)) << 2));
-                acc[4 * k + 0] = fmaf(wt[s], v4.x, acc[4 * k + 0]);
-                acc[4 * k + 1] = fmaf(wt[s], v4.y, acc[4 * k + 1]);
-                acc[4 * k + 2] = fmaf(wt[s], v4.z, acc[4 * k + 2]);
-                acc[4 * k + 3] = fmaf(wt[s], v4.w, acc[4 * k + 3]);
-              }
+            for (int k = 0; k < 8; ++k) {
+              const float4 v4 = *reinterpret_cast<const float4*>(row + (((cg * 8 + k) ^ (lr & 7)) << 2));
+              acc[4 * k + 0] = fmaf(wt, v4.x, acc[4 * k + 0]);
+              acc[4 * k + 1] = fmaf(wt, v4.y, acc[4 * k + 1]);
+              acc[4 * k + 2] = fmaf(wt, v4.z, acc[4 * k + 2]);
+              acc[4 * k + 3] = fmaf(wt, v4.w, acc[4 * k + 3]);
             }
           }
           const float inv = 1.f / L;

@@ -40,7 +40,8 @@ struct kvc_ctx {
   std::vector<Prof> prof;
   // KVC_FLAG_ASYNC_COMPRESS: the side stream, per layer an event after its attention and one after its
   // compress kernel, and whether that compress may still be running (host objects, created on first use)
-  cudaStream_t side;
+  static constexpr int kSideStreams = 2;     // layers alternate between them: consecutive compress kernels may overlap
+  cudaStream_t side[kSideStreams];
   std::vector<cudaEvent_t> ev_attn, ev_comp;
   std::vector<char> pending;
   char err[512];
@@ -109,7 +110,7 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->encode = nullptr;
   c->use_tc = cfg->dtype == KVC_BF16 && !(cfg->flags & KVC_FLAG_CUDA_CORES);
   c->profiling = false;
-  c->side = nullptr;
+  for (auto& s : c->side) s = nullptr;
   c->pending.assign(cfg->n_layers, 0);
   c->err[0] = 0;
   *out = c;
@@ -168,15 +169,21 @@ static int wait_pending(kvc_ctx* c, int l0, int l1, cudaStream_t st) {
 }
 
 static int ensure_side_stream(kvc_ctx* c) {
-  if (c->side) return KVC_OK;
-  cudaError_t e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
-  if (e != cudaSuccess) { c->side = nullptr; return fail(c, KVC_ECUDA, "cudaStreamCreate: %s", cudaGetErrorString(e)); }
-  c->ev_attn.assign(c->cfg.n_layers, nullptr);
-  c->ev_comp.assign(c->cfg.n_layers, nullptr);
+  if (c->side[0]) return KVC_OK;                             // set last: marks a complete set of events and streams
+  cudaError_t e = cudaSuccess;
+  c->ev_attn.resize(c->cfg.n_layers, nullptr);
+  c->ev_comp.resize(c->cfg.n_layers, nullptr);
   for (int l = 0; l < c->cfg.n_layers; ++l) {
-    if ((e = cudaEventCreateWithFlags(&c->ev_attn[l], cudaEventDisableTiming)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&c->ev_comp[l], cudaEventDisableTiming)) != cudaSuccess)
-      return fail(c, KVC_ECUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+    if (!c->ev_attn[l] && (e = cudaEventCreateWithFlags(&c->ev_attn[l], cudaEventDisableTiming)) != cudaSuccess) c->ev_attn[l] = nullptr;
+    if (e == cudaSuccess && !c->ev_comp[l] && (e = cudaEventCreateWithFlags(&c->ev_comp[l], cudaEventDisableTiming)) != cudaSuccess) c->ev_comp[l] = nullptr;
+    if (e != cudaSuccess) return fail(c, KVC_ECUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+  }
+  for (int i = kvc_ctx::kSideStreams - 1; i >= 0; --i) {
+    if (c->side[i]) continue;
+    if ((e = cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking)) != cudaSuccess) {
+      c->side[i] = nullptr;
+      return fail(c, KVC_ECUDA, "cudaStreamCreate: %s", cudaGetErrorString(e));
+    }
   }
   return KVC_OK;
 }
@@ -188,12 +195,12 @@ extern "C" int kvc_join(kvc_ctx* c, void* stream) {
 
 extern "C" int kvc_destroy(kvc_ctx* c) {
   if (!live(c)) return KVC_ESTATE;
-  if (c->side) {
-    cudaStreamSynchronize(c->side);
+  {
+    for (auto s : c->side) if (s) cudaStreamSynchronize(s);
     for (auto ev : c->ev_attn) if (ev) cudaEventDestroy(ev);
     for (auto ev : c->ev_comp) if (ev) cudaEventDestroy(ev);
-    cudaStreamDestroy(c->side);
-    c->side = nullptr;
+    c->ev_attn.clear(); c->ev_comp.clear();
+    for (auto& s : c->side) { if (s) cudaStreamDestroy(s); s = nullptr; }
   }
   drop_events(c);
   c->magic = 0;
@@ -586,9 +593,9 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (evict) {
     if (async_compress) {
       if (int rc = ensure_side_stream(c)) return rc;
-      if ((e = cudaEventRecord(c->ev_attn[layer0], st)) != cudaSuccess || (e = cudaStreamWaitEvent(c->side, c->ev_attn[layer0], 0)) != cudaSuccess)
+      if ((e = cudaEventRecord(c->ev_attn[layer0], st)) != cudaSuccess || (e = cudaStreamWaitEvent(c->side[layer0 % kvc_ctx::kSideStreams], c->ev_attn[layer0], 0)) != cudaSuccess)
         return check_cuda(c, e, "side stream fork");
-      st = c->side;                                           // everything below goes to the side stream
+      st = c->side[layer0 % kvc_ctx::kSideStreams];                                           // everything below goes to the side stream
     }
     const bool pdl = pdl_main && !async_compress;             // an event, not a kernel, precedes the side stream's launches
     const bool keydiff = cf.policy == KVC_SCORE_KEYDIFF;      // query-agnostic: always scored inside the fused kernel

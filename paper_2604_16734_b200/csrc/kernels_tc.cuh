@@ -159,8 +159,38 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       }
     } else if (warp == 9 || (warp == 10 && has_B)) {
       // ---------------------------------------------------------------- MMA issuer of tile t
+      // a0 append (Alg. 1: C <- C u (K_i, V_i)).  The block's keys and values pass through the ring as key tiles
+      // anyway: the issuer of tile A stores such a tile from its ring slot into cache rows n_c + 128u .. with one
+      // TMA store per 64 columns (rows past the block are zero in the tile and land in unused cache rows or are
+      // clipped at cap).  Among the CTAs that load block tile u, the one whose rows contain token 128u owns it.
+      // Nobody in this kernel reads the appended rows.  The lanes of the warp write the positions.
+      const int u_lo = max(t_begin, Tc) - Tc, u_hi = t_end - Tc;            // block tiles of this CTA: [u_lo, u_hi)
+      auto owns = [&](int u) { return (u * 128) / (2 * TOK) == pair; };
+      if (warp == 9 && u_hi > u_lo) {
+        bool waited = false;
+        for (int u = u_lo; u < u_hi; ++u) {
+          if (!owns(u)) continue;
+          if (!waited) { pdl_wait(); waited = true; }                       // the previous block's compaction is done with the cache
+          int* pos = reinterpret_cast<int*>(cache + layer * p.cache_ls + p.pos_off) + static_cast<long long>(g) * p.cap + p.n_c;
+          for (int i = u * 128 + lane; i < min(p.n, u * 128 + 128); i += 32) pos[i] = static_cast<int>(p.pos0 + i);
+        }
+      }
       if (lane == 0 && Tl > 0) {
         const int t = warp - 9;
+        bool stored = false, store_waited = false;
+        // item i of the ring (2j = K, 2j+1 = V of local key tile j) has landed in `slot`: store it if it is ours;
+        // true if the slot must not be handed back before the store has read it
+        auto append_item = [&](int i, int slot) {
+          const int u = t_begin + (i >> 1) - Tc;
+          if (t != 0 || u < 0 || !owns(u)) return false;
+          if (!store_waited) { pdl_wait(); store_waited = true; }
+          const CUtensorMap* tm = (i & 1) ? &tm_v : &tm_k;
+          for (int sub = 0; sub < NSUB; ++sub)
+            tma_store_4d(tm, ring + slot * TILE_BYTES + sub * kSubTileBytes, sub * 64, p.n_c + u * 128, g, layer);
+          tma_store_commit();
+          stored = true;
+          return i + kStages < 2 * Tl;
+        };
         constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
         constexpr uint32_t hi = smem_desc_hi_sw128(1024);
@@ -192,6 +222,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           tc_fence_after_sync();
           issue_S(0, s_cols(0));
           mma_commit(s_bar(0));
+          if (append_item(0, 0)) tma_store_wait_read();
           mma_commit(&sh.kv_empty[0]);
         }
         if (ok && dbuf && Tl > 1) {                  // K_1 sits in ring slot 2
@@ -200,6 +231,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             tc_fence_after_sync();
             issue_S(2, s_cols(1));
             mma_commit(s_bar(1));
+            if (append_item(2, 2)) tma_store_wait_read();
             mma_commit(&sh.kv_empty[2]);
           }
         }
@@ -211,11 +243,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           if (!ok) break;
           tc_fence_after_sync();
           issue_PV(slotV, 0, j > 0, s_cols(j));
+          const bool hold_v = append_item(iv, slotV);
           ok = mbar_wait(&sh.p_half[t][1], j & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           issue_PV(slotV, 1, true, s_cols(j));
           mma_commit(&sh.pv_done[t]);
+          if (hold_v) tma_store_wait_read();
           mma_commit(&sh.kv_empty[slotV]);
           if (jn < Tl) {
             ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
@@ -223,9 +257,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             tc_fence_after_sync();
             issue_S(slotK, s_cols(jn));              // overwrites P of tile jn - 2, whose P V is queued ahead of it
             mma_commit(s_bar(jn));
+            if (append_item(ik, slotK)) tma_store_wait_read();
             mma_commit(&sh.kv_empty[slotK]);
           }
         }
+        if (stored) tma_store_wait_all();            // the appended rows are in the cache before the kernel ends
       }
     }
     __syncwarp();
@@ -247,40 +283,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     float m_ref = -INFINITY, l = 0.f;                        // reference maximum (log2 units) and row sum
     bool ok = true;
     const bool active = t == 0 || has_B;
-    if (t == 1) {
-      // ---------------------------------------------------------------- a0 append (Alg. 1: C <- C u (K_i, V_i))
-      // Nobody in this kernel reads the appended rows (the block's keys come from the inputs), so the 128
-      // threads of tile B -- idle until tile A has had its first turn, or for the whole kernel when there
-      // is no tile B -- copy this CTA's share of the block's keys, values and positions into cache rows
-      // n_c .. tot.  The CTAs of a kv-head share the rows.
-      pdl_wait();                                            // the previous block's compaction is done with the cache
-      char* blob = cache + layer * p.cache_ls;
-      constexpr int VEC = D * 2 / 16;                        // 16-byte pieces per row (K or V)
-      constexpr int RPS = 128 / (2 * VEC);                   // rows per step of the 128 threads
-      constexpr int UNROLL = 4;                              // loads in flight per thread
-      const int sub = (threadIdx.x - 128) / (2 * VEC), piece = threadIdx.x % (2 * VEC);
-      const bool is_v = piece >= VEC;
-      const __nv_bfloat16* src_base = (is_v ? v_in : k_in) + layer * p.kv_ls;
-      char* dst_base = blob + (is_v ? p.v_off : 0);
-      const int stride = gridDim.x * RPS;
-      for (int t0 = blockIdx.x * RPS + sub; t0 < p.n; t0 += stride * UNROLL) {
-        uint4 val[UNROLL];
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-          const int tk = t0 + u * stride;
-          if (tk < p.n) val[u] = reinterpret_cast<const uint4*>(src_base + (static_cast<long long>(tk) * p.Hkv + g) * D)[piece % VEC];
-        }
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-          const int tk = t0 + u * stride;
-          if (tk < p.n) {
-            const long long dst_row = static_cast<long long>(g) * p.cap + p.n_c + tk;
-            reinterpret_cast<uint4*>(dst_base + dst_row * D * 2)[piece % VEC] = val[u];
-            if (piece == 0) reinterpret_cast<int*>(blob + p.pos_off)[dst_row] = static_cast<int>(p.pos0 + tk);
-          }
-        }
-      }
-    }
     // Turn taking (named barrier 2 + t = "tile t may go", 128 waiters + 128 arrivals).  Tile A goes first.
     const bool turns = has_B && Tl > 0;
     if (turns && t == 1) named_barrier_arrive(2, 256);

@@ -35,8 +35,9 @@ static constexpr int kStages = 4;                 // K/V ring slots of the atten
 // The two softmax groups take turns on the exponentials (named barriers): while one tile's exponentials
 // occupy the CUDA cores the tensor pipe runs the other tile's MMAs; without the hand-over both tiles fall
 // into lockstep and the two pipes idle alternately.  Loading S and finding the maxima is outside the turn.
-// (Measured and dropped: eight softmax warps per row tile, two threads per row -- no faster, the per-tile
-// chain is not bound by the instruction count per thread.)
+// (Measured and dropped: eight softmax warps per row tile, two threads per row, also in the form where a CTA
+// with a single row tile lends it the other tile's warps -- no faster, the per-tile chain is not bound by the
+// instruction count per thread; and a polynomial 2^x on the FMA pipe for part of the columns -- slower.)
 // TMEM columns: S_A/P_A [0,128)  S_B/P_B [128,256)  O_A [256,384)  O_B [384,512).
 // The running output is rescaled lazily: a row keeps its reference maximum until the true maximum
 // has grown by more than 2^8, so P stays below 256 and O rarely needs touching.
@@ -360,6 +361,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           }
           tmem_st16(tmem_S + c * 16, pk);
           if (c & 1) {                                        // 64 keys of P are in TMEM: release them to the MMA warp
+            // With alternating S buffers this tile's S was queued two tiles ago, so nothing else ties the softmax
+            // threads to the issuer's progress: they wait (long over by now) for P V of the previous tile, and can
+            // never be two rounds ahead on p_half, which a parity wait could not tell apart.
+            if (dbuf && c == 1 && j > 0) {
+              ok = __all_sync(0xffffffffu, mbar_wait(&sh.pv_done[t], (j - 1) & 1, abort_flag));
+              if (!ok) break;
+            }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&sh.p_half[t][c >> 1]);

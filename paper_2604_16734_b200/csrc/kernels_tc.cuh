@@ -64,8 +64,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
                                                                    const __grid_constant__ CUtensorMap tm_v,
                                                                    const __grid_constant__ CUtensorMap tm_kin,
                                                                    const __grid_constant__ CUtensorMap tm_vin,
-                                                                   const __nv_bfloat16* __restrict__ k_in,
-                                                                   const __nv_bfloat16* __restrict__ v_in,
                                                                    char* __restrict__ cache,
                                                                    __nv_bfloat16* __restrict__ out,
                                                                    char* __restrict__ ws, Geom p, int S) {

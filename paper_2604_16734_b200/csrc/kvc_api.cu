@@ -38,7 +38,7 @@ struct kvc_ctx {
   bool profiling;
   struct Prof { int kind; cudaEvent_t a, b; };
   std::vector<Prof> prof;
-  // KVC_FLAG_ASYNC_COMPRESS: the side stream, per layer an event after its attention and one after its
+  // KVC_FLAG_ASYNC_COMPRESS: the side streams, per layer an event after its attention and one after its
   // compress kernel, and whether that compress may still be running (host objects, created on first use)
   static constexpr int kSideStreams = 2;     // layers alternate between them: consecutive compress kernels may overlap
   cudaStream_t side[kSideStreams];
@@ -390,8 +390,8 @@ static int attn_key_splits(const Geom& g) {
 
 template <int D>
 static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                  const CUtensorMap& tkin, const CUtensorMap& tvin, const void* k, const void* v, void* cache,
-                                  void* out, void* ws, int S, bool pdl, cudaStream_t st) {
+                                  const CUtensorMap& tkin, const CUtensorMap& tvin, void* cache, void* out, void* ws, int S,
+                                  bool pdl, cudaStream_t st) {
   const int smem = (2 + kvc::kStages) * (D / 64) * kvc::kSubTileBytes + 1024;
   static bool attr_set = false;
   if (!attr_set) {
@@ -410,8 +410,8 @@ static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CU
   LaunchAttrs la(S, pdl);
   lc.attrs = la.at;
   lc.numAttrs = la.n;
-  return cudaLaunchKernelEx(&lc, kvc::attn_tc_kernel<D>, tq, tk, tv, tkin, tvin, (const __nv_bfloat16*)k,
-                            (const __nv_bfloat16*)v, (char*)cache, (__nv_bfloat16*)out, (char*)ws, g, S);
+  return cudaLaunchKernelEx(&lc, kvc::attn_tc_kernel<D>, tq, tk, tv, tkin, tvin, (char*)cache, (__nv_bfloat16*)out,
+                            (char*)ws, g, S);
 }
 // a2..a4 fused (compress.cuh).  MODE: kvc::kScoresGiven / kScoreAttention / kScoreKeyDiff.
 template <int D, int MODE>
@@ -580,8 +580,8 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   ProfScope ps(c, 1, st);
   if (c->use_tc) {
     const int S = (cf.flags & 4u) ? 1 : attn_key_splits(g);
-    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, tkin, tvin, k, v, cache, out, ws, S, pdl, st)
-                 : launch_tc_attn<64>(g, tq, tk, tv, tkin, tvin, k, v, cache, out, ws, S, pdl, st);
+    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, pdl, st)
+                 : launch_tc_attn<64>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, pdl, st);
   } else if (f32) {
     if (D == 128) launch_cc_attn<float, 128>(g, q, cache, out, ws, st); else launch_cc_attn<float, 64>(g, q, cache, out, ws, st);
   } else {

@@ -30,8 +30,7 @@ static constexpr int kStages = 4;                 // K/V ring slots of the atten
 //               (64 keys each) so the first PV MMAs start while the second half of the exponentials
 //               is still being computed.
 //   warp  11    only gives its registers away (setmaxnreg works on groups of four warps)
-// a0: before their first turn the threads of tile B copy the CTA's share of the block's keys, values and
-// positions into the cache.
+// a0: the block's key / value tiles are stored into the cache from their ring slots (TMA stores issued by warp 9).
 // The two softmax groups take turns on the exponentials (named barriers): while one tile's exponentials
 // occupy the CUDA cores the tensor pipe runs the other tile's MMAs; without the hand-over both tiles fall
 // into lockstep and the two pipes idle alternately.  Loading S and finding the maxima is outside the turn.
@@ -129,6 +128,22 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       if (lane == 0) {
         tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
         tma_prefetch_desc(&tm_kin); tma_prefetch_desc(&tm_vin);
+      }
+      // While the previous kernel drains: ask L2 for the Q tiles and the first two key / value tiles (a hint only,
+      // nothing is read into the SM before the wait below), so that the first loads find them there.
+      if (Tl > 0 && lane < 2 + 2 * NSUB * min(Tl, 2)) {
+        if (lane < 2) {
+          if (lane == 0 || has_B)
+            for (int sub = 0; sub < NSUB; ++sub) tma_prefetch_l2_4d(&tm_q, sub * 64, g * p.G, lane ? tokB : tokA, layer);
+        } else {
+          const int i = (lane - 2) / NSUB, sub = (lane - 2) % NSUB;      // ring item i: K or V of key tile t_begin + i/2
+          const int kt = t_begin + (i >> 1);
+          if (kt < Tc) tma_prefetch_l2_4d((i & 1) ? &tm_v : &tm_k, sub * 64, kt * 128, g, layer);
+          else tma_prefetch_l2_4d((i & 1) ? &tm_vin : &tm_kin, sub * 64, g, (kt - Tc) * 128, layer);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) {
         pdl_wait();                                // the block's keys were appended by the previous kernel
       }
       if (lane == 0 && Tl > 0) {

@@ -78,6 +78,15 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, ui
       : "memory");
 }
 
+// Hint: bring one box of a tensor into L2.  No data reaches the SM and nothing is ordered by it, so it may be
+// issued before the data's producer is known to have finished (L2 is the point of coherence: a later write
+// updates the line).  Same alignment rule as the load.
+__device__ __forceinline__ void tma_prefetch_l2_4d(const void* tmap, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+               ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
+}
+
 // TMA store of one box from shared memory (bulk async-group completion).  Coordinates past the tensor's extent
 // are clipped.  The innermost coordinate must be a multiple of 16 bytes, the others are free.
 __device__ __forceinline__ void tma_store_4d(const void* tmap, const void* smem_src, int c0, int c1, int c2, int c3) {

@@ -222,7 +222,8 @@ def test_random_small_configurations(seed):
     B = max(B, w)
     c = rnd.choice([40, 128, 150, 260])
     policy = rnd.choice(["attn", "attn", "keydiff"])
-    kvc = Kvc(1, hq, hkv, d, dtype, B, c, w, policy=binding.KVC_SCORE_KEYDIFF if policy == "keydiff" else 0)
+    kvc = Kvc(1, hq, hkv, d, dtype, B, c, w, policy=binding.KVC_SCORE_KEYDIFF if policy == "keydiff" else 0,
+              flags=KVC_FLAG_ASYNC_COMPRESS if seed % 2 else 0)          # odd seeds: compress on the side streams
     orc = KVCOracle(1, hq, hkv, d, B, w, policy=policy)
     torch.manual_seed(seed)
     p = 0

@@ -46,7 +46,10 @@ static constexpr int kStages = 4;                 // K/V ring slots of the atten
 // distributed shared memory: rank s owns rows [s*128/S, (s+1)*128/S) of both tiles, every CTA copies
 // its partial rows (fp32) into the owner's shared memory with remote stores, the cluster
 // synchronises, and each rank combines and writes its rows.  Nothing but the final result goes to HBM.
-// grid (ceil(ceil(n/TOK)/2) * S, Hkv, nl), cluster (S,1,1), block 384,
+// Row tiles per CTA: R = 2 as described, or R = 1 (tile A only; S then alternates between both tiles' TMEM columns):
+// a CTA with one row tile runs its key tiles about 0.7 times as fast per row tile, but exchanges half as much in
+// the combine and doubles the CTA count, which lets a launch that would need S = 4 do with S = 2; the host picks.
+// grid (ceil(ceil(n/TOK)/R) * S, Hkv, nl), cluster (S,1,1), block 384,
 // dynamic smem (2 + kStages) * (D/64) * 16 KB + 1 KB.
 static constexpr int kAttnThreads = 384;
 
@@ -65,7 +68,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
                                                                    const __grid_constant__ CUtensorMap tm_vin,
                                                                    char* __restrict__ cache,
                                                                    __nv_bfloat16* __restrict__ out,
-                                                                   char* __restrict__ ws, Geom p, int S) {
+                                                                   char* __restrict__ ws, Geom p, int S, int R) {
   constexpr int NSUB = D / 64;
   constexpr int TILE_BYTES = NSUB * kSubTileBytes;
   constexpr uint32_t TMEM_COLS = 512;
@@ -78,12 +81,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
 
   const int layer = blockIdx.z, g = blockIdx.y;
   const int split = S > 1 ? static_cast<int>(cluster_ctarank()) : 0;
-  const int pair = blockIdx.x / S;
+  const int pair = blockIdx.x / S;               // index of this CTA's group of R row tiles (R = 1 or 2)
   const int TOK = 128 / p.G, rows = TOK * p.G;
-  const int tokA = pair * 2 * TOK, tokB = tokA + TOK;
-  const bool has_B = tokB < p.n;
+  const int tokA = pair * R * TOK, tokB = tokA + TOK;
+  const bool has_B = R == 2 && tokB < p.n;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int last_tok = min(tokA + 2 * TOK, p.n) - 1;
+  const int last_tok = min(tokA + R * TOK, p.n) - 1;
   // Key tiles this pair of row tiles can see: Tc tiles of the cache (rows [0, n_c), the last one possibly
   // partial), then the block's own keys in tiles of 128 tokens, read straight from the k/v inputs.
   const int Tc = (p.n_c + 127) / 128;
@@ -91,7 +94,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
   const int t_begin = split * T / S, t_end = (split + 1) * T / S;
   const int Tl = t_end - t_begin;                // key tiles of this CTA (0 is possible when S > T)
 
-  pdl_launch_dependents();                       // the next kernel of the stream may set itself up meanwhile
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.q_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.pv_done[i], 1);
@@ -179,7 +181,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       // clipped at cap).  Among the CTAs that load block tile u, the one whose rows contain token 128u owns it.
       // Nobody in this kernel reads the appended rows.  The lanes of the warp write the positions.
       const int u_lo = max(t_begin, Tc) - Tc, u_hi = t_end - Tc;            // block tiles of this CTA: [u_lo, u_hi)
-      auto owns = [&](int u) { return (u * 128) / (2 * TOK) == pair; };
+      auto owns = [&](int u) { return (u * 128) / (R * TOK) == pair; };
       if (warp == 9 && u_hi > u_lo) {
         bool waited = false;
         for (int u = u_lo; u < u_hi; ++u) {
@@ -391,6 +393,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         if (turns && !took_turn) named_barrier(2 + t, 256);   // a wait gave up before the turn was taken: take it now
         if (turns && !(t == 1 && j + 1 == Tl)) named_barrier_arrive(3 - t, 256);
       }
+      // The key loop is over: the next kernel of the stream may be scheduled and set itself up while this one
+      // writes its results.  (Triggered at the start instead, the waiting CTAs of the next attention launch take the
+      // SMs that the compress kernel of the previous layer, ready on a side stream, could use.)
+      if (threadIdx.x == 0) pdl_launch_dependents();
       if (ok && Tl > 0) ok = mbar_wait(&sh.pv_done[t], (Tl - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);                       // the TMEM accesses below are warp-wide
       if (ok && Tl > 0) tc_fence_after_sync();

@@ -376,22 +376,37 @@ struct LaunchAttrs {
 // (An exchange of the partials through an L2-resident global buffer instead of distributed shared
 // memory was measured too: slower, the release / acquire round trip costs more than the narrow
 // SM-to-SM path.)
-static int attn_key_splits(const Geom& g) {
+// Launch shape of the tensor-core attention: R row tiles per CTA (1 or 2) and the key split S over a cluster.
+// For each R the split is the largest that the SM count, the portable cluster size and the rule of three key
+// tiles per CTA allow; the two candidates are then compared with a model of the kernel's duration fitted to
+// in-kernel time stamps (us): a key tile costs 2.1 per pair of row tiles taking turns and 1.45 for a single
+// tile; the combine costs 3.5 for its barriers and the reduce plus 3.6 per row tile for the remote stores of a
+// whole tile's partial rows; CTAs beyond one per SM run as further waves.
+static void attn_launch_shape(const Geom& g, bool allow_split, int* S_out, int* R_out) {
   const int TOK = 128 / g.G;
-  const int pairs = ((g.n + TOK - 1) / TOK + 1) / 2;
-  const long long base = (long long)pairs * g.Hkv * g.nl;
+  const int tiles = (g.n + TOK - 1) / TOK;
   const int T = (g.n_c + 127) / 128 + (g.n + 127) / 128;
-  int S = (int)(kvc::kNumSMs / base);
-  if (S > 8) S = 8;                    // portable cluster size limit
-  if (S > T / 3) S = T / 3;            // the exchange costs about as much as two key tiles: keep three per CTA
-  while (S & (S - 1)) S &= S - 1;      // a power of two: the 128 rows of a tile divide evenly among the ranks
-  return S < 1 ? 1 : S;
+  double best = 0.0;
+  for (int R = 2; R >= 1; --R) {
+    const long long base = (long long)((tiles + R - 1) / R) * g.Hkv * g.nl;
+    int S = allow_split ? (int)(kvc::kNumSMs / base) : 1;
+    if (S > 8) S = 8;                    // portable cluster size limit
+    if (S > T / 3) S = T / 3;            // the exchange costs about as much as two key tiles: keep three per CTA
+    while (S & (S - 1)) S &= S - 1;      // a power of two: the 128 rows of a tile divide evenly among the ranks
+    if (S < 1) S = 1;
+    const int Tl = (T + S - 1) / S;
+    const long long waves = (base * S + kvc::kNumSMs - 1) / kvc::kNumSMs;
+    double est = Tl * (R == 2 ? 2.1 : 1.45) * (double)waves;
+    if (S > 1) est += 3.5 + R * 3.6 * (S - 1) / S;
+    if (R == 2 || est < best) { best = est; *S_out = S; *R_out = R; }
+    if (tiles == 1) break;               // a single row tile: both shapes are the same launch
+  }
 }
 
 template <int D>
 static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                   const CUtensorMap& tkin, const CUtensorMap& tvin, void* cache, void* out, void* ws, int S,
-                                  bool pdl, cudaStream_t st) {
+                                  int R, bool pdl, cudaStream_t st) {
   const int smem = (2 + kvc::kStages) * (D / 64) * kvc::kSubTileBytes + 1024;
   static bool attr_set = false;
   if (!attr_set) {
@@ -400,10 +415,10 @@ static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CU
     attr_set = true;
   }
   const int TOK = 128 / g.G;
-  const int pairs = ((g.n + TOK - 1) / TOK + 1) / 2;
+  const int groups = ((g.n + TOK - 1) / TOK + R - 1) / R;
   cudaLaunchConfig_t lc;
   memset(&lc, 0, sizeof(lc));
-  lc.gridDim = dim3(pairs * S, g.Hkv, g.nl);
+  lc.gridDim = dim3(groups * S, g.Hkv, g.nl);
   lc.blockDim = dim3(kvc::kAttnThreads, 1, 1);
   lc.dynamicSmemBytes = smem;
   lc.stream = st;
@@ -411,7 +426,7 @@ static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CU
   lc.attrs = la.at;
   lc.numAttrs = la.n;
   return cudaLaunchKernelEx(&lc, kvc::attn_tc_kernel<D>, tq, tk, tv, tkin, tvin, (char*)cache, (__nv_bfloat16*)out,
-                            (char*)ws, g, S);
+                            (char*)ws, g, S, R);
 }
 // a2..a4 fused (compress.cuh).  MODE: kvc::kScoresGiven / kScoreAttention / kScoreKeyDiff.
 template <int D, int MODE>
@@ -579,9 +594,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   {
   ProfScope ps(c, 1, st);
   if (c->use_tc) {
-    const int S = (cf.flags & 4u) ? 1 : attn_key_splits(g);
-    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, pdl, st)
-                 : launch_tc_attn<64>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, pdl, st);
+    int S = 1, R = 2;
+    attn_launch_shape(g, !(cf.flags & 4u), &S, &R);
+    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st)
+                 : launch_tc_attn<64>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st);
   } else if (f32) {
     if (D == 128) launch_cc_attn<float, 128>(g, q, cache, out, ws, st); else launch_cc_attn<float, 64>(g, q, cache, out, ws, st);
   } else {

@@ -93,6 +93,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
   const int T = Tc + (last_tok + 128) / 128;
   const int t_begin = split * T / S, t_end = (split + 1) * T / S;
   const int Tl = t_end - t_begin;                // key tiles of this CTA (0 is possible when S > T)
+  // A CTA with one row tile and at least two key tiles runs the tile twice over: softmax group and issuer t take the
+  // key tiles t, t+2, ... with accumulators, maxima and sums of their own (the TMEM columns of tile B are free), two
+  // key tiles are in flight as with two row tiles, and the two partial results are merged at the end.
+  const bool alt = !has_B && Tl >= 2;
+  const int n_it[2] = {alt ? (Tl + 1) / 2 : Tl, alt ? Tl / 2 : (has_B ? Tl : 0)};   // key tiles of group 0 / 1
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -173,7 +178,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           }
         }
       }
-    } else if (warp == 9 || (warp == 10 && has_B)) {
+    } else if (warp == 9 || (warp == 10 && (has_B || alt))) {
       // ---------------------------------------------------------------- MMA issuer of tile t
       // a0 append (Alg. 1: C <- C u (K_i, V_i)).  The block's keys and values pass through the ring as key tiles
       // anyway: the issuer of tile A stores such a tile from its ring slot into cache rows n_c + 128u .. with one
@@ -194,11 +199,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       if (lane == 0 && Tl > 0) {
         const int t = warp - 9;
         bool stored = false, store_waited = false;
-        // item i of the ring (2j = K, 2j+1 = V of local key tile j) has landed in `slot`: store it if it is ours;
+        // item i of the ring (2j = K, 2j+1 = V of local key tile j) has landed in `slot`: store it if it is ours
+        // (with two row tiles the issuer of tile A stores, else the issuer that consumes the item);
         // true if the slot must not be handed back before the store has read it
         auto append_item = [&](int i, int slot) {
           const int u = t_begin + (i >> 1) - Tc;
-          if (t != 0 || u < 0 || !owns(u)) return false;
+          if ((t != 0 && !alt) || u < 0 || !owns(u)) return false;
           if (!store_waited) { pdl_wait(); store_waited = true; }
           const CUtensorMap* tm = (i & 1) ? &tm_v : &tm_k;
           for (int sub = 0; sub < NSUB; ++sub)
@@ -210,16 +216,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
         constexpr uint32_t hi = smem_desc_hi_sw128(1024);
-        const uint32_t q_lo = smem_desc_lo(smem_u32(sQ) + t * TILE_BYTES, 16);          // K-major operand
+        const uint32_t q_lo = smem_desc_lo(smem_u32(sQ) + (alt ? 0 : t) * TILE_BYTES, 16);   // K-major operand
         const uint32_t k_lo0 = smem_desc_lo(smem_u32(ring), 16);                        // K-major operand
         const uint32_t v_lo0 = smem_desc_lo(smem_u32(ring), kSubTileBytes);             // MN-major operand
-        const uint32_t tO = tmem + 256 + t * 128;
-        // A CTA with one row tile has the other tile's S columns to spare: S alternates between the two buffers, and
-        // S of key tile j+1 is queued before P V of tile j, so that the softmax threads find it waiting.
-        const bool dbuf = !has_B;
-        auto s_cols = [&](int j) { return tmem + (dbuf ? (j & 1) : t) * 128; };
-        auto s_bar = [&](int j) { return &sh.s_full[dbuf ? (j & 1) : t]; };
-        auto issue_S = [&](int slot, uint32_t tS) {  // S_t = Q_t K^T, 16 of the d columns per MMA
+        const uint32_t tS = tmem + t * 128, tO = tmem + 256 + t * 128;
+        const int first = alt ? t : 0, step = alt ? 2 : 1;   // local key tiles of this issuer: first, first + step, ...
+        auto issue_S = [&](int slot) {               // S_t = Q_t K^T, 16 of the d columns per MMA
           const uint32_t k_lo = k_lo0 + slot * (TILE_BYTES >> 4);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
@@ -227,43 +229,34 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             mma_ss_lh(tS, q_lo + off, hi, k_lo + off, hi, idesc_qk, kk > 0);
           }
         };
-        auto issue_PV = [&](int slot, int half, bool acc, uint32_t tS) {   // O_t += P_t V, 16 keys per MMA, 64 keys per half
+        auto issue_PV = [&](int slot, int half, bool acc) {   // O_t += P_t V, 16 keys per MMA, 64 keys per half
           const uint32_t v_lo = v_lo0 + slot * (TILE_BYTES >> 4);
 #pragma unroll
           for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
             mma_ts_lh(tO, tS + kk * 8, v_lo + kk * (2048 >> 4), hi, idesc_pv, acc || kk > 0);
         };
-        bool ok = mbar_wait(&sh.q_full[t], 0, abort_flag) && mbar_wait(&sh.kv_full[0], 0, abort_flag);
+        const int i0 = 2 * first;                    // ring item of this issuer's first K tile (slot i0, first round)
+        bool ok = mbar_wait(&sh.q_full[alt ? 0 : t], 0, abort_flag) && mbar_wait(&sh.kv_full[i0], 0, abort_flag);
         if (ok) {
           tc_fence_after_sync();
-          issue_S(0, s_cols(0));
-          mma_commit(s_bar(0));
-          if (append_item(0, 0)) tma_store_wait_read();
-          mma_commit(&sh.kv_empty[0]);
+          issue_S(i0);
+          mma_commit(&sh.s_full[t]);
+          if (append_item(i0, i0)) tma_store_wait_read();
+          mma_commit(&sh.kv_empty[i0]);
         }
-        if (ok && dbuf && Tl > 1) {                  // K_1 sits in ring slot 2
-          ok = mbar_wait(&sh.kv_full[2], 0, abort_flag);
-          if (ok) {
-            tc_fence_after_sync();
-            issue_S(2, s_cols(1));
-            mma_commit(s_bar(1));
-            if (append_item(2, 2)) tma_store_wait_read();
-            mma_commit(&sh.kv_empty[2]);
-          }
-        }
-        for (int j = 0; j < Tl && ok; ++j) {
-          const int jn = dbuf ? j + 2 : j + 1;       // the key tile whose S is queued behind P V of tile j
-          const int iv = 2 * j + 1, ik = 2 * jn;
+        for (int jj = first, it = 0; jj < Tl && ok; jj += step, ++it) {
+          const int jn = jj + step;                  // the key tile whose S is queued behind P V of this one
+          const int iv = 2 * jj + 1, ik = 2 * jn;
           const int slotV = iv % kStages, slotK = ik % kStages;
-          ok = mbar_wait(&sh.p_half[t][0], j & 1, abort_flag) && mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
+          ok = mbar_wait(&sh.p_half[t][0], it & 1, abort_flag) && mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          issue_PV(slotV, 0, j > 0, s_cols(j));
+          issue_PV(slotV, 0, it > 0);
           const bool hold_v = append_item(iv, slotV);
-          ok = mbar_wait(&sh.p_half[t][1], j & 1, abort_flag);
+          ok = mbar_wait(&sh.p_half[t][1], it & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          issue_PV(slotV, 1, true, s_cols(j));
+          issue_PV(slotV, 1, true);
           mma_commit(&sh.pv_done[t]);
           if (hold_v) tma_store_wait_read();
           mma_commit(&sh.kv_empty[slotV]);
@@ -271,8 +264,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
-            issue_S(slotK, s_cols(jn));              // overwrites P of tile jn - 2, whose P V is queued ahead of it
-            mma_commit(s_bar(jn));
+            issue_S(slotK);
+            mma_commit(&sh.s_full[t]);
             if (append_item(ik, slotK)) tma_store_wait_read();
             mma_commit(&sh.kv_empty[slotK]);
           }
@@ -290,26 +283,25 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     // ---------------------------------------------------------------- softmax + epilogue of tile t
     const int t = warp >> 2;
     const int r = (warp & 3) * 32 + lane;                     // row of the tile = TMEM lane
-    const int tok0 = t ? tokB : tokA;
+    const int tok0 = (t && !alt) ? tokB : tokA;             // (both groups hold the rows of tile A when they alternate)
     const int tok = tok0 + r / p.G, hh = r % p.G;
     const bool row_valid = r < rows && tok < p.n;
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t tmem_O = tmem + 256 + t * 128 + lane_addr;
-    const bool dbuf = !has_B;                                // one row tile: S alternates between both tiles' columns
+    const uint32_t tmem_S = tmem + t * 128 + lane_addr, tmem_O = tmem + 256 + t * 128 + lane_addr;
     float m_ref = -INFINITY, l = 0.f;                        // reference maximum (log2 units) and row sum
     bool ok = true;
-    const bool active = t == 0 || has_B;
-    // Turn taking (named barrier 2 + t = "tile t may go", 128 waiters + 128 arrivals).  Tile A goes first.
-    const bool turns = has_B && Tl > 0;
+    const bool writer = t == 0 || has_B;                     // this group writes results (a row tile of its own)
+    const bool active = writer || alt;                       // this group takes part in the key loop
+    const int first = alt ? t : 0, step = alt ? 2 : 1;       // local key tiles of this group: first, first + step, ...
+    // Turn taking (named barrier 2 + t = "group t may go", 128 waiters + 128 arrivals).  Group 0 goes first.
+    const bool turns = (has_B || alt) && Tl > 0;
     if (turns && t == 1) named_barrier_arrive(2, 256);
     if (active) {
-      for (int j = 0; j < Tl; ++j) {
-        const int kt = t_begin + j;                           // key tile index
+      for (int jj = first, it = 0; jj < Tl; jj += step, ++it) {
+        const int kt = t_begin + jj;                          // key tile index
         // Waits that gave up only skip the arithmetic: the turn barrier is passed on every path, once per key
         // tile and warp, so the other row tile never waits for a turn that is not handed over.
-        const uint32_t tmem_S = tmem + (dbuf ? (j & 1) : t) * 128 + lane_addr;
-        if (ok) ok = __all_sync(0xffffffffu, dbuf ? mbar_wait(&sh.s_full[j & 1], (j >> 1) & 1, abort_flag)
-                                                  : mbar_wait(&sh.s_full[t], j & 1, abort_flag));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[t], it & 1, abort_flag));
         bool took_turn = false;
         if (ok) do {
         tc_fence_after_sync();
@@ -337,14 +329,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         const float mx = fmaxf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])),
                                fmaxf(fmaxf(mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
         const float m_new = mx * p.scale_log2;                // scale > 0
-        if (j == 0) {
+        if (it == 0) {
           m_ref = m_new == -INFINITY ? 0.f : m_new;
         } else {
           const bool grow = m_new > m_ref + kRescaleThreshold;
           if (__any_sync(0xffffffffu, grow)) {
             const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;
             if (grow) { m_ref = m_new; l *= f; }
-            ok = __all_sync(0xffffffffu, mbar_wait(&sh.pv_done[t], (j - 1) & 1, abort_flag));   // O_t holds every earlier tile
+            ok = __all_sync(0xffffffffu, mbar_wait(&sh.pv_done[t], (it - 1) & 1, abort_flag));  // O_t holds every earlier tile
             if (!ok) break;
             tc_fence_after_sync();
 #pragma unroll
@@ -376,13 +368,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           }
           tmem_st16(tmem_S + c * 16, pk);
           if (c & 1) {                                        // 64 keys of P are in TMEM: release them to the MMA warp
-            // With alternating S buffers this tile's S was queued two tiles ago, so nothing else ties the softmax
-            // threads to the issuer's progress: they wait (long over by now) for P V of the previous tile, and can
-            // never be two rounds ahead on p_half, which a parity wait could not tell apart.
-            if (dbuf && c == 1 && j > 0) {
-              ok = __all_sync(0xffffffffu, mbar_wait(&sh.pv_done[t], (j - 1) & 1, abort_flag));
-              if (!ok) break;
-            }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&sh.p_half[t][c >> 1]);
@@ -391,16 +376,65 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
         } while (0);
         if (turns && !took_turn) named_barrier(2 + t, 256);   // a wait gave up before the turn was taken: take it now
-        if (turns && !(t == 1 && j + 1 == Tl)) named_barrier_arrive(3 - t, 256);
+        // hand the turn over if the other group has a key tile left: its it-th (group 0 asks) or (it+1)-th (group 1)
+        if (turns && (t == 0 ? it < n_it[1] : it + 1 < n_it[0])) named_barrier_arrive(3 - t, 256);
       }
       // The key loop is over: the next kernel of the stream may be scheduled and set itself up while this one
       // writes its results.  (Triggered at the start instead, the waiting CTAs of the next attention launch take the
       // SMs that the compress kernel of the previous layer, ready on a side stream, could use.)
       if (threadIdx.x == 0) pdl_launch_dependents();
-      if (ok && Tl > 0) ok = mbar_wait(&sh.pv_done[t], (Tl - 1) & 1, abort_flag);
+      if (ok && n_it[t] > 0) ok = mbar_wait(&sh.pv_done[t], (n_it[t] - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);                       // the TMEM accesses below are warp-wide
-      if (ok && Tl > 0) tc_fence_after_sync();
-      if (S == 1) {
+      if (ok && n_it[t] > 0) tc_fence_after_sync();
+      if (alt) {
+        // Merge the two groups' partial results into group 0's accumulator: group 1 parks its rows of O (fp32, 16-byte
+        // chunks XOR-swizzled with row & 7 against bank conflicts) and (m, l) in shared memory over the Q tiles, which
+        // nobody reads once both groups are past their last P V; group 0 rescales both to the common maximum.
+        float* mrg = reinterpret_cast<float*>(smem);          // [128][D]
+        named_barrier(5, 256);
+        if (t == 1) {
+          if (ok) {
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[32];
+              tmem_ld32(tmem_O + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 8; ++k)
+                *reinterpret_cast<uint4*>(mrg + r * D + (((c * 8 + k) ^ (r & 7)) << 2)) = make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+            }
+          }
+          sh.stat[2 * r] = (ok && l > 0.f) ? m_ref : -INFINITY;   // -inf: this group saw no key of the row
+          sh.stat[2 * r + 1] = l;
+        }
+        named_barrier(5, 256);
+        if (t == 0 && ok) {
+          const float m1 = sh.stat[2 * r], l1 = sh.stat[2 * r + 1];
+          if (__any_sync(0xffffffffu, m1 != -INFINITY)) {
+            const float m_all = fmaxf(m_ref, m1);              // group 0 has seen key tile 0, hence a key of every row
+            const float w0 = fast_exp2(m_ref - m_all), w1 = m1 == -INFINITY ? 0.f : fast_exp2(m1 - m_all);
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[32];
+              tmem_ld32(tmem_O + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const float4 b4 = *reinterpret_cast<const float4*>(mrg + r * D + (((c * 8 + k) ^ (r & 7)) << 2));
+                o[4 * k + 0] = __float_as_uint(fmaf(w1, b4.x, w0 * __uint_as_float(o[4 * k + 0])));
+                o[4 * k + 1] = __float_as_uint(fmaf(w1, b4.y, w0 * __uint_as_float(o[4 * k + 1])));
+                o[4 * k + 2] = __float_as_uint(fmaf(w1, b4.z, w0 * __uint_as_float(o[4 * k + 2])));
+                o[4 * k + 3] = __float_as_uint(fmaf(w1, b4.w, w0 * __uint_as_float(o[4 * k + 3])));
+              }
+              tmem_st32(tmem_O + c * 32, o);
+            }
+            tmem_wait_st();
+            l = fmaf(w1, l1, w0 * l);
+            m_ref = m_all;
+          }
+        }
+      }
+      if (S == 1 && writer) {
         if (ok) {
           const float inv = 1.f / l;
           __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D;
@@ -446,7 +480,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       float* stat = sh.stat;                                    // [S][2][rows_per][2]: m (-inf: row saw no key), l
       cluster_arrive();                                         // every CTA is done with its Q tiles and ring
       cluster_wait();
-      if (active) {
+      if (writer) {
         const int nthr = has_B ? 256 : 128;                     // softmax threads that take part
         const bool have = ok && Tl > 0;                         // warp-uniform
         for (int tt = 0; tt < (has_B ? 2 : 1); ++tt) {

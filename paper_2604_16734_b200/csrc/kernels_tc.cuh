@@ -386,8 +386,62 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       if (ok && n_it[t] > 0) ok = mbar_wait(&sh.pv_done[t], (n_it[t] - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);                       // the TMEM accesses below are warp-wide
       if (ok && n_it[t] > 0) tc_fence_after_sync();
-      if (alt) {
-        // Merge the two groups' partial results into group 0's accumulator: group 1 parks its rows of O (fp32, 16-byte
+      if (alt && S == 1) {
+        // Merge and write out, half the columns per group: group t keeps columns [t*D/2, (t+1)*D/2) of its O in
+        // registers and parks the other half (fp32, 16-byte chunks XOR-swizzled with row & 7 against bank conflicts)
+        // and its (m, l) in shared memory over the Q tiles, which nobody reads once both groups are past their
+        // last P V; then each group combines its columns of both partial results and writes them.
+        constexpr int H = D / 2;
+        float* mrg = reinterpret_cast<float*>(smem);          // [2 groups][128][H]
+        named_barrier(5, 256);
+        if (ok) {
+#pragma unroll
+          for (int c = 0; c < H / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_O + (1 - t) * H + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              *reinterpret_cast<uint4*>(mrg + (t * 128 + r) * H + (((c * 8 + k) ^ (r & 7)) << 2)) = make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+          }
+        }
+        sh.stat[(t * 128 + r) * 2] = (ok && l > 0.f) ? m_ref : -INFINITY;   // -inf: this group saw no key of the row
+        sh.stat[(t * 128 + r) * 2 + 1] = l;
+        named_barrier(5, 256);
+        if (ok) {
+          const float m1 = sh.stat[((1 - t) * 128 + r) * 2], l1 = sh.stat[((1 - t) * 128 + r) * 2 + 1];
+          const float m0 = l > 0.f ? m_ref : -INFINITY;
+          const float m_all = fmaxf(m0, m1);                   // finite: group 0 has seen key tile 0, hence a key of every row
+          const float w0 = fast_exp2(m0 - m_all), w1 = fast_exp2(m1 - m_all);
+          const float L = fmaf(w1, l1, w0 * l);
+          const float inv = 1.f / L, a0 = w0 * inv, a1 = w1 * inv;
+          __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D + t * H;
+#pragma unroll
+          for (int c = 0; c < H / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_O + t * H + c * 32, o);
+            tmem_wait_ld();
+            if (row_valid) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float4 b0 = *reinterpret_cast<const float4*>(mrg + ((1 - t) * 128 + r) * H + (((c * 8 + 2 * i) ^ (r & 7)) << 2));
+                const float4 b1 = *reinterpret_cast<const float4*>(mrg + ((1 - t) * 128 + r) * H + (((c * 8 + 2 * i + 1) ^ (r & 7)) << 2));
+                uint4 vv;
+                vv.x = pack_bf16x2(fmaf(a1, b0.x, a0 * __uint_as_float(o[8 * i + 0])), fmaf(a1, b0.y, a0 * __uint_as_float(o[8 * i + 1])));
+                vv.y = pack_bf16x2(fmaf(a1, b0.z, a0 * __uint_as_float(o[8 * i + 2])), fmaf(a1, b0.w, a0 * __uint_as_float(o[8 * i + 3])));
+                vv.z = pack_bf16x2(fmaf(a1, b1.x, a0 * __uint_as_float(o[8 * i + 4])), fmaf(a1, b1.y, a0 * __uint_as_float(o[8 * i + 5])));
+                vv.w = pack_bf16x2(fmaf(a1, b1.z, a0 * __uint_as_float(o[8 * i + 6])), fmaf(a1, b1.w, a0 * __uint_as_float(o[8 * i + 7])));
+                reinterpret_cast<uint4*>(orow + c * 32)[i] = vv;
+              }
+            }
+          }
+          if (row_valid && t == 0) {
+            float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
+            lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_all + log2f(L)) * 0.6931471805599453f;
+          }
+        }
+      } else if (alt) {
+        // Key split: merge the two groups' partial results into group 0's accumulator for the cluster combine below: group 1 parks its rows of O (fp32, 16-byte
         // chunks XOR-swizzled with row & 7 against bank conflicts) and (m, l) in shared memory over the Q tiles, which
         // nobody reads once both groups are past their last P V; group 0 rescales both to the common maximum.
         float* mrg = reinterpret_cast<float*>(smem);          // [128][D]
@@ -434,7 +488,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           }
         }
       }
-      if (S == 1 && writer) {
+      if (S == 1 && writer && !alt) {
         if (ok) {
           const float inv = 1.f / l;
           __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D;

@@ -324,14 +324,16 @@ def test_compress_on_side_stream_matches_in_order_compress(name, units, n_layers
     a = _kvc_for(cfg); b = _kvc_for(cfg, KVC_FLAG_ASYNC_COMPRESS)
     out_a = torch.zeros_like(Q); out_b = torch.zeros_like(Q)
 
-    def run(kvc, out):
+    def run(kvc, out, join=True):
         kvc.reset()
         for pos0, n in cfg.chunks():
             for l in range(n_layers):
                 kvc.prefill_chunk(l, Q[l, pos0:pos0 + n], K[l, pos0:pos0 + n], V[l, pos0:pos0 + n], pos0, out[l, pos0:pos0 + n])
-        kvc.join()
+        if join:
+            kvc.join()
 
     run(a, out_a)
+    run(b, out_b, join=False)        # the next request's reset has to order itself after the pending compress kernels
     run(b, out_b)
     torch.cuda.synchronize()
     if graph:

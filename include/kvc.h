@@ -160,14 +160,17 @@ int kvc_prefill_chunk_layers(kvc_ctx* ctx, int layer0, int n_layers, const void*
                              size_t cache_layer_stride, void* workspace, void* out,
                              long long out_layer_stride, void* stream);
 
-/* Bytes of the DEVICE staging buffer kvc_prefill_chunk_host needs (room for q, k, v and out of a
- * block of max(max_chunk, B) tokens). */
+/* Bytes of the DEVICE staging buffer kvc_prefill_chunk_host needs (two halves, each with room for q, k, v
+ * and out of a block of max(max_chunk, B) tokens). */
 int kvc_staging_nbytes(const kvc_ctx* ctx, size_t* nbytes);
 
 /* kvc_prefill_chunk with HOST q/k/v/out (pinned memory recommended): copies the block's q, k, v
  * into `staging` (DEVICE, kvc_staging_nbytes bytes, 256-byte aligned), runs the block, copies `out`
- * back to the host.  Everything is asynchronous on `stream`; out_host is valid after the stream
- * is synchronised. */
+ * back to the host.  Nothing blocks the host; out_host is valid, and the host inputs may be reused, after
+ * `stream` is synchronised.  Consecutive calls alternate between the two halves of `staging`: the
+ * host-to-device copies of a call run on a stream the context owns and `stream` waits for them, so they
+ * overlap the previous call's kernels and device-to-host copy (pass the same `staging` to every call of a
+ * context; a run-time error before the kernels leaves the call without effect on the cache). */
 int kvc_prefill_chunk_host(kvc_ctx* ctx, int layer, const void* q_host, const void* k_host,
                            const void* v_host, int n, long long pos0, void* cache, void* workspace,
                            void* staging, void* out_host, void* stream);

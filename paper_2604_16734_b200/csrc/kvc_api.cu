@@ -44,6 +44,11 @@ struct kvc_ctx {
   cudaStream_t side[kSideStreams];
   std::vector<cudaEvent_t> ev_attn, ev_comp;
   std::vector<char> pending;
+  // kvc_prefill_chunk_host: the stream that carries the host-to-device copies, per staging half an event after its
+  // copies (recorded there) and one after the block that read it (recorded on the caller's stream); call counter
+  cudaStream_t copy_in;
+  cudaEvent_t ev_in[2], ev_free[2];
+  unsigned host_calls;
   char err[512];
 };
 
@@ -112,6 +117,9 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->profiling = false;
   for (auto& s : c->side) s = nullptr;
   c->pending.assign(cfg->n_layers, 0);
+  c->copy_in = nullptr;
+  for (int i = 0; i < 2; ++i) { c->ev_in[i] = nullptr; c->ev_free[i] = nullptr; }
+  c->host_calls = 0;
   c->err[0] = 0;
   *out = c;
   return KVC_OK;
@@ -201,6 +209,12 @@ extern "C" int kvc_destroy(kvc_ctx* c) {
     for (auto ev : c->ev_comp) if (ev) cudaEventDestroy(ev);
     c->ev_attn.clear(); c->ev_comp.clear();
     for (auto& s : c->side) { if (s) cudaStreamDestroy(s); s = nullptr; }
+    if (c->copy_in) { cudaStreamSynchronize(c->copy_in); cudaStreamDestroy(c->copy_in); c->copy_in = nullptr; }
+    for (int i = 0; i < 2; ++i) {
+      if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+      if (c->ev_free[i]) cudaEventDestroy(c->ev_free[i]);
+      c->ev_in[i] = c->ev_free[i] = nullptr;
+    }
   }
   drop_events(c);
   c->magic = 0;
@@ -674,13 +688,31 @@ extern "C" int kvc_prefill_chunk_layers(kvc_ctx* c, int layer0, int n_layers, co
                    workspace, out, out_layer_stride, (cudaStream_t)stream);
 }
 
+// q, k, v and out of one block, each rounded up to 256 bytes
+static size_t staging_half_bytes(size_t qb, size_t kb) { return 2 * align_up(qb, 256) + 2 * align_up(kb, 256); }
+
 extern "C" int kvc_staging_nbytes(const kvc_ctx* c, size_t* nbytes) {
   if (!live(c)) return KVC_ESTATE;
   if (!nbytes) return KVC_EINVAL;
   const size_t rows = c->cfg.max_chunk > c->cfg.budget ? c->cfg.max_chunk : c->cfg.budget;   // room for a bulk first block
   const size_t qb = rows * c->cfg.n_q_heads * c->cfg.head_dim * c->elem;
   const size_t kb = rows * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
-  *nbytes = 2 * align_up(qb, 256) + 2 * align_up(kb, 256);
+  *nbytes = 2 * staging_half_bytes(qb, kb);                  // two halves: the copies of one block run beside the previous block
+  return KVC_OK;
+}
+
+static int ensure_copy_stream(kvc_ctx* c) {
+  if (c->copy_in) return KVC_OK;                             // set last: marks a complete set
+  cudaError_t e = cudaSuccess;
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    if (!c->ev_in[i] && (e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming)) != cudaSuccess) c->ev_in[i] = nullptr;
+    if (e == cudaSuccess && !c->ev_free[i] && (e = cudaEventCreateWithFlags(&c->ev_free[i], cudaEventDisableTiming)) != cudaSuccess) c->ev_free[i] = nullptr;
+  }
+  if (e != cudaSuccess) return fail(c, KVC_ECUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+  if ((e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking)) != cudaSuccess) {
+    c->copy_in = nullptr;
+    return fail(c, KVC_ECUDA, "cudaStreamCreate: %s", cudaGetErrorString(e));
+  }
   return KVC_OK;
 }
 
@@ -696,16 +728,27 @@ extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host,
   cudaStream_t st = (cudaStream_t)stream;
   const size_t qb = (size_t)n * c->cfg.n_q_heads * c->cfg.head_dim * c->elem;
   const size_t kb = (size_t)n * c->cfg.n_kv_heads * c->cfg.head_dim * c->elem;
-  char* dq = (char*)staging;
+  size_t total = 0;
+  kvc_staging_nbytes(c, &total);
+  int rc = ensure_copy_stream(c);
+  if (rc) return rc;
+  // Calls alternate between the two halves of the staging buffer.  The inputs travel on the context's copy stream,
+  // behind the block that last read this half (two calls ago), so they overlap the previous call's kernels and its
+  // device-to-host copy; the caller's stream waits for them, runs the block and copies `out` back.
+  const int half = (int)(c->host_calls++ & 1u);
+  char* dq = (char*)staging + half * (total / 2);
   char* dk = dq + align_up(qb, 256);
   char* dv = dk + align_up(kb, 256);
   char* dout = dv + align_up(kb, 256);
-  int rc;
-  if ((rc = check_cuda(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st), "H2D q"))) return rc;
-  if ((rc = check_cuda(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, st), "H2D k"))) return rc;
-  if ((rc = check_cuda(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, st), "H2D v"))) return rc;
+  if ((rc = check_cuda(c, cudaStreamWaitEvent(c->copy_in, c->ev_free[half], 0), "cudaStreamWaitEvent"))) return rc;
+  if ((rc = check_cuda(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, c->copy_in), "H2D q"))) return rc;
+  if ((rc = check_cuda(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, c->copy_in), "H2D k"))) return rc;
+  if ((rc = check_cuda(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, c->copy_in), "H2D v"))) return rc;
+  if ((rc = check_cuda(c, cudaEventRecord(c->ev_in[half], c->copy_in), "cudaEventRecord"))) return rc;
+  if ((rc = check_cuda(c, cudaStreamWaitEvent(st, c->ev_in[half], 0), "cudaStreamWaitEvent"))) return rc;
   rc = run_chunk(c, layer, 1, dq, 0, dk, dv, 0, n, pos0, cache, 0, workspace, dout, 0, st, 0, false);   // staging is reused: no side stream
   if (rc) return rc;
+  if ((rc = check_cuda(c, cudaEventRecord(c->ev_free[half], st), "cudaEventRecord"))) return rc;
   return check_cuda(c, cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st), "D2H out");
 }
 

@@ -235,6 +235,24 @@ def test_random_small_configurations(seed):
         p += n - t
 
 
+@pytest.mark.parametrize("hkv,G,d,B,c,flags", [(1, 1, 128, 3100, 128, 0), (2, 4, 128, 2100, 200, KVC_FLAG_ASYNC_COMPRESS),
+                                               (1, 8, 64, 1500, 384, 0)])
+def test_deep_key_split(hkv, G, d, B, c, flags):
+    # few (kv-head, row tile) pairs and a long cache: the key range is split over clusters of up to eight CTAs, the
+    # CTAs with a single row tile run it as two alternating halves, and the block's tiles are appended by whichever
+    # CTA owns them; the first call fills the cache in one pass (hybrid schedule)
+    from oracle.kvc_oracle import KVCOracle
+    hq = hkv * G
+    kvc = Kvc(1, hq, hkv, d, torch.bfloat16, B, c, 32, flags=flags)
+    orc = KVCOracle(1, hq, hkv, d, B, 32)
+    torch.manual_seed(B + c)
+    p = 0
+    for n in (B, c, c - 1, c // 2 + 1):
+        q = torch.randn(n, hq, d).bfloat16(); k = (torch.randn(n, hkv, d) + 0.3).bfloat16(); v = torch.randn(n, hkv, d).bfloat16()
+        compare_chunk(kvc, orc, 0, q, k, v, p)
+        p += n
+
+
 def test_first_block_larger_than_budget_and_window_equal_to_budget():
     torch.manual_seed(8)
     hq, hkv, d = 4, 2, 128

@@ -206,7 +206,7 @@ def test_ragged_blocks(dtype, d, hq, hkv, flags):
         p += n
 
 
-@pytest.mark.parametrize("seed", list(range(12)))
+@pytest.mark.parametrize("seed", list(range(24)))
 def test_random_small_configurations(seed):
     # random shapes, budgets, windows, block lengths, policies and proxy counts against the oracle
     import random

@@ -64,6 +64,7 @@ def load_peaks():
 NCU_TRAFFIC = {
     "sources": "a7a040cee37801b6",
     "bytes_per_launch": {("C2", "attention"): 7411712, ("C2", "compress"): 4203008,
+                         ("C4", "attention"): 10883584, ("C4", "compress"): 5417984,
                          ("C5", "attention"): 29738240, ("C5", "compress"): 12622592},
 }
 

@@ -1,8 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the block-wise prefill hot path (append, attention, score, select, compact).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--mode graph|direct|batched]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C5] [--mode graph|direct|batched]
   python bench.py --impl reference ...      # the CPU oracle as the reference arm
+
+The default workload is C5 (long video), the largest single-GPU configuration and the one in which a launch
+carries enough work for the roofline targets to be assessed.  At N = 1 the same JSON line carries, under
+"workloads", the other bf16 configurations (C2, C3, C4 and the block-size study's T4), each measured the same way
+with fewer steps (--no-extra skips them).
 
 One "step" is one pass of the whole hot path over one synthetic request: every block of the
 workload's prefix through every layer, starting from empty caches.  Prints ONE JSON line.
@@ -57,16 +62,11 @@ def load_peaks():
 
 
 # ------------------------------------------------------------------------------------------------
-# DRAM traffic of one steady-state launch (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture,
-# summarised under profiles/), valid only for the kernel sources it was taken from: the hash below is that
-# of the CUDA sources at capture time, and the figure is reported as null once they have changed.
+# DRAM traffic of one steady-state launch (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture),
+# kept as text under profiles/ together with a hash of the CUDA sources it was taken from; it is reported as
+# null once the sources have changed.  File format: a line "sources <hash>", then "<workload> <kernel> <bytes>".
 
-NCU_TRAFFIC = {
-    "sources": "a7a040cee37801b6",
-    "bytes_per_launch": {("C2", "attention"): 7411712, ("C2", "compress"): 4203008,
-                         ("C4", "attention"): 10883584, ("C4", "compress"): 5417984,
-                         ("C5", "attention"): 29738240, ("C5", "compress"): 12622592},
-}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")
 
 
 def kernel_sources_hash():
@@ -85,9 +85,16 @@ def kernel_sources_hash():
 
 
 def ncu_traffic(workload, kernel):
-    if kernel_sources_hash() != NCU_TRAFFIC["sources"]:
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    except OSError:
         return None
-    return NCU_TRAFFIC["bytes_per_launch"].get((workload, kernel))
+    table = {(r[0], r[1]): int(r[2]) for r in rows if len(r) == 3}
+    src = next((r[1] for r in rows if len(r) == 2 and r[0] == "sources"), None)
+    if src != kernel_sources_hash():
+        return None
+    return table.get((workload, kernel))
 
 
 # ------------------------------------------------------------------------------------------------
@@ -225,14 +232,24 @@ def cpu_threads():
         return os.cpu_count() or 1
 
 
+def config_dict(cfg, L, args, world, extra=None):
+    """The `config` object of the JSON line: the same keys for both arms."""
+    d = {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+         "head_dim": cfg.head_dim, "tokens": cfg.n_tokens, "block": cfg.chunk, "budget": cfg.budget,
+         "obs_window": cfg.obs_window, "policy": args.policy, "schedule": "hybrid" if args.hybrid else "block-wise",
+         "proxy_tokens": args.proxy, "mode": args.mode, "parallelism": f"replicas x{world}"}
+    if extra:
+        d.update(extra)
+    return d
+
+
 def reference_arm(args, cfg, rank):
     if rank != 0:
         return
-    import numpy as np
     wl = Workload(cfg, device="cpu")
     q, k, v = wl.layer(0)
     tens = (q.double().numpy(), k.double().numpy(), v.double().numpy())
-    for _ in range(min(args.warmup, 1)):
+    for _ in range(args.warmup):
         run_oracle_sample(cfg, tens)
     vals, times = [], []
     desc = ""
@@ -240,10 +257,12 @@ def reference_arm(args, cfg, rank):
         val, dt, desc = run_oracle_sample(cfg, tens)
         vals.append(val); times.append(dt)
     value = sum(vals) / len(vals)
+    L = args.layers if args.layers else cfg.n_layers
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "sample": desc},
+            "config": config_dict(cfg, L, args, int(os.environ.get("WORLD_SIZE", "1")),
+                                  {"compress": "n/a (CPU oracle)", "l2": "n/a (CPU oracle)", "sample": desc}),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -419,13 +438,188 @@ def profile_pass(r: Runner, steps: int, batched: bool = False):
     return per
 
 
+def rates(per, peaks):
+    for d in per.values():
+        sec = d["ms_total_per_step"] / 1e3
+        d["gbs"] = d["bytes_per_step"] / sec / 1e9
+        d["tflops"] = d["flops_per_step"] / sec / 1e12
+        d["hbm_frac"] = d["gbs"] / peaks["hbm_gbs"]
+        d["tensor_frac_sustained"] = d["tflops"] / peaks["tflops_sustained"]
+        d["tensor_frac_burst"] = d["tflops"] / peaks["tflops_burst"]
+    return per
+
+
+def step_roofline(cfg, per, L, ms_per_step, peaks):
+    """The path's roofline for one step (all blocks x L layers), from the exact algorithmic work of the step: the
+    slower of the attention at the measured bf16 peak (its own HBM time where that is longer, or its HBM time alone
+    for fp32, which does not use the tensor cores) and the score / select / compact bytes at the measured HBM
+    bandwidth; also the stricter sum of the two, since the steps of one layer run back to back."""
+    att = per.get("attention")
+    if not att:
+        return None
+    hbm = peaks["hbm_gbs"] * 1e9
+    t_att_hbm = (att["bytes_per_step"] + per.get("append", {}).get("bytes_per_step", 0)) / hbm
+    t_att_tc = att["flops_per_step"] / (peaks["tflops_sustained"] * 1e12) if cfg.dtype == "bf16" else 0.0
+    t_att = max(t_att_hbm, t_att_tc)
+    t_cmp = sum(per[s]["bytes_per_step"] for s in ("score", "compress") if s in per) / hbm
+    bound, bound_sum = max(t_att, t_cmp), t_att + t_cmp
+    meas = ms_per_step / 1e3
+    return dict(bound_ms=1e3 * bound, bound_sum_ms=1e3 * bound_sum, measured_ms=ms_per_step, frac=bound / meas,
+                frac_of_sum_bound=bound_sum / meas,
+                attention_bound="tensor" if t_att_tc >= t_att_hbm else "hbm", attention_ms_at_peak=1e3 * t_att,
+                compress_ms_at_hbm=1e3 * t_cmp,
+                tokens_per_s_per_layer_at_bound=cfg.n_tokens * L / bound,
+                peak_source=peaks["source"] + " (sustained bf16, copy bandwidth)")
+
+
+def measure(cfg, args, L, local_rank, rank, world, dist, barrier, peaks, steps, primary):
+    """Times one workload: the step as configured (`value`), the same step with every kernel in stream order, the
+    kernels one by one, and (primary workload only) the end-to-end path from host buffers and the CPU oracle."""
+    flags = args.flags
+    side_stream = (args.mode != "batched" and not args.sync_compress and cfg.dtype == "bf16" and not flags & 1)
+    if side_stream:
+        flags |= 16
+    r = Runner(cfg, local_rank, L, flags, 1 if args.policy == "keydiff" else 0, args.hybrid, args.proxy)
+    kv = r.kvc
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    step = {"direct": r.step_direct, "batched": r.step_batched, "graph": r.step_graph}[args.mode]
+    (r.step_batched if args.mode == "batched" else r.step_direct)()   # sets function attributes, resolves the driver entry point
+    torch.cuda.synchronize()
+    if args.mode == "graph":
+        r.capture()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert kv.status() == 0, kv.last_error()
+    launches_before = kv.launch_count()
+    if args.mode == "graph":              # a replay launches what one captured step launched
+        r.step_direct(); torch.cuda.synchronize()
+        launches_per_step = kv.launch_count() - launches_before
+    secs, t0, t1 = time_steps(step, steps, barrier)
+    if args.mode != "graph":
+        launches_per_step = (kv.launch_count() - launches_before) // steps
+    assert kv.status() == 0, kv.last_error()
+    secs = max_over_ranks(secs, dist, "cuda")
+    rows = sampler.stop()
+    clocks = sampler.summary(rows, t0, t1)
+    value = whole_job_value(cfg.n_tokens, L, steps, world, secs)
+    ms_per_step = 1e3 * secs / steps
+    out = dict(value=value, ms_per_step=ms_per_step, steps=steps, launches_per_step=launches_per_step, clocks=clocks)
+
+    # ---- the same step with every kernel in stream order (no side streams): the serial chain of the launches
+    in_order_ms = None
+    if rank == 0 and not args.no_profile:
+        if side_stream and args.mode in ("graph", "direct"):
+            saved = (r.kvc, r.flags, r.graph)
+            r.kvc, r.flags = r.kvc_in_order, r.flags & ~16
+            r.step_direct(); torch.cuda.synchronize()
+            if args.mode == "graph":
+                r.capture()
+            fn = r.step_graph if args.mode == "graph" else r.step_direct
+            for _ in range(2):
+                fn()
+            n_io = max(3, min(steps, 10))
+            io_secs, _, _ = time_steps(fn, n_io, lambda: None)
+            in_order_ms = 1e3 * io_secs / n_io
+            r.kvc, r.flags, r.graph = saved
+        else:
+            in_order_ms = ms_per_step
+        out["ms_per_step_in_order"] = in_order_ms
+
+    # ---- per-kernel durations and rooflines (rank 0, outside the timed region)
+    per, per_b, roof = {}, {}, None
+    if rank == 0 and not args.no_profile:
+        per = rates(profile_pass(r, max(3, min(steps, 10)) if primary else 3), peaks)
+        ridge = peaks["tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+        dom = max(per, key=lambda s: per[s]["ms_total_per_step"])
+        d = per[dom]
+        ai = d["flops_per_step"] / max(d["bytes_per_step"], 1)
+        if cfg.dtype == "bf16" and dom == "attention" and ai > ridge:
+            # the kernel is timed inside a long step: the sustained peak is its denominator; the burst figure beside it
+            roof = dict(kernel=dom, bound="tensor", achieved=d["tflops"], peak=peaks["tflops_sustained"], unit="TFLOP/s",
+                        frac=d["tflops"] / peaks["tflops_sustained"], traffic=None,
+                        peak_source=peaks["source"] + " (sustained bf16)", peak_burst=peaks["tflops_burst"],
+                        frac_of_burst_peak=d["tflops"] / peaks["tflops_burst"])
+        else:
+            roof = dict(kernel=dom, bound="hbm", achieved=d["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=d["gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"])
+        roof["traffic"] = ncu_traffic(cfg.name, dom) if L == cfg.n_layers else None
+        roof["algorithmic_bytes_per_launch"] = d["bytes_per_step"] / max(d["launches_per_step"], 1)
+        roof["algorithmic_flops_per_launch"] = d["flops_per_step"] / max(d["launches_per_step"], 1)
+        roof["us_per_launch"] = d["us_per_launch"]
+        roof["arithmetic_intensity"] = ai
+        roof["timing"] = "CUDA events around every launch on the launching stream, every kernel alone on the GPU"
+        # the kernels' event-timed durations against the step they have to fit into
+        kernel_ms_sum = sum(x["ms_total_per_step"] for x in per.values())
+        out["kernel_ms_sum"] = kernel_ms_sum
+        out["overlap"] = dict(
+            ms_per_step_in_order=in_order_ms, ms_per_step=ms_per_step,
+            hidden_by_side_streams_ms=(in_order_ms - ms_per_step) if in_order_ms is not None else None,
+            kernel_ms_sum_over_in_order=kernel_ms_sum / in_order_ms if in_order_ms else None,
+            note="kernel_ms_sum brackets every launch with an event pair (a few us each, no overlap between "
+                 "consecutive launches); in the in-order step consecutive launches overlap through programmatic "
+                 "dependent launch")
+        out["roofline_step"] = step_roofline(cfg, per, L, ms_per_step, peaks)
+        if in_order_ms is not None and out["roofline_step"]:
+            out["roofline_step"]["frac_in_order"] = out["roofline_step"]["bound_ms"] / in_order_ms
+        # ---- the same kernels with all layers in one launch (possible only with synthetic inputs): what the
+        #      bandwidth-bound steps reach when a launch carries enough bytes to fill the GPU
+        if L > 1 and not args.proxy:
+            per_b = rates(profile_pass(r, 3, batched=True), peaks)
+    out["kernels"], out["kernels_layer_batched"], out["roofline"] = per, per_b, roof
+
+    # ---- end to end through the host-buffer entry point
+    if primary and not args.no_e2e and not args.proxy:          # (the host-buffer entry point has no proxy variant)
+        host = tuple(t.cpu().pin_memory() for t in (r.Q, r.K, r.V)) + (torch.empty(r.O.shape, dtype=r.O.dtype).pin_memory(),)
+        for _ in range(2):
+            r.step_host(host)
+        torch.cuda.synchronize()
+        e_steps = max(1, min(steps, 5))
+        esecs, _, _ = time_steps(lambda: r.step_host(host), e_steps, barrier)
+        esecs = max_over_ranks(esecs, dist, "cuda")
+        h2d = sum(t.numel() * t.element_size() for t in host[:3])
+        d2h = host[3].numel() * host[3].element_size()
+        out["e2e"] = dict(value=world * cfg.n_tokens * L * e_steps / esecs, unit=UNIT, h2d_bytes_per_step=h2d,
+                          d2h_bytes_per_step=d2h, steps=e_steps, ms_per_step=1e3 * esecs / e_steps)
+        del host
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
+    if primary and rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # the same bounded sample on successive layers until about 10 s of CPU work have been spent
+        tot_dt, vals, desc, nl_done = 0.0, [], "", 0
+        while nl_done < L and tot_dt < 10.0:
+            tens = tuple(t[nl_done].double().cpu().numpy() for t in (r.Q, r.K, r.V))
+            val, dt, desc = run_oracle_sample(cfg, tens)
+            vals.append(val); tot_dt += dt; nl_done += 1
+        out["cpu_baseline"] = dict(value=len(vals) / sum(1.0 / x for x in vals), unit=UNIT, cores=cpu_threads(), kind="oracle",
+                                   sample=desc.replace("layer 0", f"layers 0..{nl_done - 1}"), seconds=tot_dt)
+
+    logical, physical, full = kv.kv_bytes(cfg.n_tokens)
+    out["kv_bytes"] = {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,
+                       "blobs_incl_positions": kv.blob_bytes * L}
+    out["config"] = config_dict(cfg, L, args, world, {
+        "compress": "side stream, beside the next layer's attention" if flags & 16 else "in stream order",
+        "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"})
+    r.kvc.close()
+    if r.kvc_in_order is not r.kvc:
+        r.kvc_in_order.close()
+    del r
+    torch.cuda.empty_cache()
+    return out
+
+
+EXTRA_WORKLOADS = ("C2", "C3", "C4", "T4")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C2", choices=sorted(CONFIGS))
+    ap.add_argument("--workload", default="C5", choices=sorted(CONFIGS))
     ap.add_argument("--mode", default="graph", choices=["graph", "direct", "batched"])
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (0 = all; not a headline run)")
     ap.add_argument("--block", type=int, default=0, help="override the workload's block size b (block-size study, Sec. 5 / Table 4)")
@@ -444,6 +638,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other workloads reported under \"workloads\"")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -473,121 +668,35 @@ def main():
     L = args.layers if args.layers else cfg.n_layers
     if args.proxy and (args.mode == "batched"):
         raise SystemExit("--proxy runs in the graph and direct modes only")
-    side_stream = (args.mode != "batched" and not args.sync_compress and cfg.dtype == "bf16" and not args.flags & 1)
-    if side_stream:
-        args.flags |= 16
-    r = Runner(cfg, local_rank, L, args.flags, 1 if args.policy == "keydiff" else 0, args.hybrid, args.proxy)
-    if args.proxy:
-        args.no_e2e = True                      # the host-buffer entry point has no proxy variant
-    kv = r.kvc
-    sampler = ClockSampler(local_rank)
-    sampler.start()
+    m = measure(cfg, args, L, local_rank, rank, world, dist, barrier, peaks, args.steps, primary=True)
 
-    step = {"direct": r.step_direct, "batched": r.step_batched, "graph": r.step_graph}[args.mode]
-    (r.step_batched if args.mode == "batched" else r.step_direct)()   # sets function attributes, resolves the driver entry point
-    torch.cuda.synchronize()
-    if args.mode == "graph":
-        r.capture()
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    assert kv.status() == 0, kv.last_error()
-    launches_before = kv.launch_count()
-    if args.mode == "graph":              # a replay launches what one captured step launched
-        r.step_direct(); torch.cuda.synchronize()
-        launches_per_step = kv.launch_count() - launches_before
-    secs, t0, t1 = time_steps(step, args.steps, barrier)
-    if args.mode != "graph":
-        launches_per_step = (kv.launch_count() - launches_before) // args.steps
-    assert kv.status() == 0, kv.last_error()
-    secs = max_over_ranks(secs, dist, "cuda")
-    tokens_layers = cfg.n_tokens * L
-    value = whole_job_value(cfg.n_tokens, L, args.steps, world, secs)
-
-    # ---- per-kernel durations and roofline (rank 0, outside the timed region)
-    per, roof = {}, None
-    if rank == 0 and not args.no_profile:
-        per = profile_pass(r, max(3, min(args.steps, 10)))
-        ridge = peaks["tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
-        for s, d in per.items():
-            sec = d["ms_total_per_step"] / 1e3
-            d["gbs"] = d["bytes_per_step"] / sec / 1e9
-            d["tflops"] = d["flops_per_step"] / sec / 1e12
-        dom = max(per, key=lambda s: per[s]["ms_total_per_step"])
-        d = per[dom]
-        ai = d["flops_per_step"] / max(d["bytes_per_step"], 1)
-        if cfg.dtype == "bf16" and dom in ("attention",) and ai > ridge:
-            roof = dict(kernel=dom, bound="tensor", achieved=d["tflops"], peak=peaks["tflops_sustained"], unit="TFLOP/s",
-                        frac=d["tflops"] / peaks["tflops_sustained"], traffic=None, peak_source=peaks["source"] + " (sustained bf16)")
-        else:
-            roof = dict(kernel=dom, bound="hbm", achieved=d["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=d["gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"])
-        roof["traffic"] = ncu_traffic(cfg.name, dom) if L == cfg.n_layers else None
-        roof["algorithmic_bytes_per_launch"] = d["bytes_per_step"] / max(d["launches_per_step"], 1)
-        roof["us_per_launch"] = d["us_per_launch"]
-        roof["arithmetic_intensity"] = ai
-
-    # ---- the same kernels with all layers in one launch (possible only with synthetic inputs): what the
-    #      bandwidth-bound steps reach when a launch carries enough bytes to fill the GPU
-    per_b = {}
-    if rank == 0 and not args.no_profile and L > 1 and not args.proxy:
-        per_b = profile_pass(r, 3, batched=True)
-        for s, d in per_b.items():
-            sec = d["ms_total_per_step"] / 1e3
-            d["gbs"] = d["bytes_per_step"] / sec / 1e9
-            d["tflops"] = d["flops_per_step"] / sec / 1e12
-            d["hbm_frac"] = d["gbs"] / peaks["hbm_gbs"]
-
-    # ---- end to end through the host-buffer entry point
-    e2e = None
-    if not args.no_e2e:
-        host = tuple(t.cpu().pin_memory() for t in (r.Q, r.K, r.V)) + (torch.empty(r.O.shape, dtype=r.O.dtype).pin_memory(),)
-        for _ in range(2):
-            r.step_host(host)
-        torch.cuda.synchronize()
-        e_steps = max(1, min(args.steps, 5))
-        esecs, _, _ = time_steps(lambda: r.step_host(host), e_steps, barrier)
-        esecs = max_over_ranks(esecs, dist, "cuda")
-        h2d = sum(t.numel() * t.element_size() for t in host[:3])
-        d2h = host[3].numel() * host[3].element_size()
-        e2e = dict(value=world * tokens_layers * e_steps / esecs, unit=UNIT, h2d_bytes_per_step=h2d,
-                   d2h_bytes_per_step=d2h, steps=e_steps, ms_per_step=1e3 * esecs / e_steps)
-        del host
-    rows = sampler.stop()
-    clocks = sampler.summary(rows, t0, t1)
-
-    # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        # the same bounded sample on successive layers until about 10 s of CPU work have been spent
-        tot_dt, vals, desc, nl_done = 0.0, [], "", 0
-        while nl_done < L and tot_dt < 10.0:
-            tens = tuple(t[nl_done].double().cpu().numpy() for t in (r.Q, r.K, r.V))
-            val, dt, desc = run_oracle_sample(cfg, tens)
-            vals.append(val); tot_dt += dt; nl_done += 1
-        cpu = dict(value=len(vals) / sum(1.0 / x for x in vals), unit=UNIT, cores=cpu_threads(), kind="oracle",
-                   sample=desc.replace("layer 0", f"layers 0..{nl_done - 1}"), seconds=tot_dt)
+    # ---- the other bf16 configurations, measured the same way (N = 1, default settings only)
+    extra = {}
+    plain = not (args.block or args.budget or args.proxy or args.hybrid or args.layers or args.flags or args.no_profile)
+    if rank == 0 and world == 1 and not args.no_extra and plain and args.policy == "attn" and args.workload == "C5":
+        for name in EXTRA_WORKLOADS:
+            c2 = CONFIGS[name]
+            x = measure(c2, args, c2.n_layers, local_rank, rank, world, None, lambda: None, peaks,
+                        max(3, min(args.steps, 10)), primary=False)
+            extra[name] = {k: x[k] for k in ("value", "ms_per_step", "ms_per_step_in_order", "steps", "launches_per_step",
+                                             "kernel_ms_sum", "kernels", "kernels_layer_batched", "roofline", "roofline_step",
+                                             "overlap", "kv_bytes", "clocks", "config") if k in x}
+            extra[name]["unit"] = UNIT
 
     if rank == 0:
-        logical, physical, full = kv.kv_bytes(cfg.n_tokens)
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-                "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-                "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
-                           "head_dim": cfg.head_dim, "tokens": cfg.n_tokens, "block": cfg.chunk, "budget": cfg.budget,
-                           "obs_window": cfg.obs_window, "policy": args.policy, "schedule": "hybrid" if args.hybrid else "block-wise", "proxy_tokens": args.proxy, "mode": args.mode,
-                           "compress": "side stream, beside the next layer's attention" if args.flags & 16 else "in stream order", "parallelism": f"replicas x{world}",
-                           "l2": "inputs exceed L2" if (r.Q.numel() + 2 * r.K.numel()) * cfg.elem_bytes > 126e6 else "inputs fit L2"},
-                "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
-                "kv_bytes": {"logical_budget": logical, "physical_allocated": physical, "uncompressed": full,
-                             "blobs_incl_positions": kv.blob_bytes * L},
-                "kernels": per, "kernels_layer_batched": per_b}
-        if roof:
-            line["roofline"] = roof
-        if e2e:
-            line["e2e"] = e2e
-        if cpu:
-            line["cpu_baseline"] = cpu
+        line = {"metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic", "config": m["config"],
+                "clocks": m["clocks"], "gpu_launches": m["launches_per_step"] * args.steps,
+                "launches_per_step": m["launches_per_step"], "kv_bytes": m["kv_bytes"], "kernels": m["kernels"],
+                "kernels_layer_batched": m["kernels_layer_batched"]}
+        for k in ("ms_per_step_in_order", "kernel_ms_sum", "overlap", "roofline_step", "e2e", "cpu_baseline"):
+            if k in m:
+                line[k] = m[k]
+        if m.get("roofline"):
+            line["roofline"] = m["roofline"]
+        if extra:
+            line["workloads"] = extra
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

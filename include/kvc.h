@@ -189,7 +189,9 @@ int kvc_prefill_chunk_host(kvc_ctx* ctx, int layer, const void* q_host, const vo
  *   - The first call on a device looks up the device address of the array (once per device, with
  *     that device current); make that first call outside any stream capture.
  *   - The array is shared by every context and every call on the device and keeps what the last
- *     call left there; the call clears the status word it needs zeroed.  Two calls whose GPU work
+ *     call left there; a call that passes its argument checks clears the status word before its
+ *     kernels run, so kvc_status_static reports on the most recent accepted call only (read it
+ *     before the next call if an earlier call's status matters).  Two calls whose GPU work
  *     overlaps (different streams, or different threads without ordering) race on it: keep all
  *     users of this entry point on one stream, or order them with events.
  *   - Calls cudaMalloc/cudaFree never, and returns KVC_ESTATE while kvc_profile_enable is on
@@ -224,6 +226,16 @@ int kvc_join(kvc_ctx* ctx, void* stream);
  * KVC_ETIMEOUT if a bounded wait inside a kernel gave up (the kernel then left early; results of
  * that call are invalid but the context and the device stay usable). */
 int kvc_status(kvc_ctx* ctx, void* workspace, void* stream);
+
+/* (No counterpart in the paper: robustness of the implementation.)  Every wait inside the kernels (on a TMA
+ * load, a tensor-core commit, another warp) is bounded; a wait that runs out makes its kernel drain and exit and
+ * leaves KVC_ETIMEOUT in the status word.  kvc_set_wait_limit sets that bound for the context's later calls, in
+ * clock cycles (default about 2e9, one second; accepted range [1024, 2^40], rounded down to a multiple of 1024).
+ * kvc_selftest_wait_timeout enqueues a one-CTA kernel whose only wait has no producer, bounded by the smaller of
+ * the context's limit and 2^21 cycles: afterwards kvc_status(workspace) returns KVC_ETIMEOUT, and the context, the
+ * device and the workspace (after kvc_workspace_init) stay usable.  workspace: DEVICE. */
+int kvc_set_wait_limit(kvc_ctx* ctx, long long cycles);
+int kvc_selftest_wait_timeout(kvc_ctx* ctx, void* workspace, void* stream);
 
 /* KV bytes after Eq. 2 (2 x layers x heads x dim_head x precision x sequence length):
  * logical uses sequence length B, physical uses cap (what the blobs really hold, pos excluded),

@@ -25,7 +25,7 @@ EXPORTS = [
     "kvc_prefill_chunk", "kvc_prefill_chunk_layers", "kvc_staging_nbytes", "kvc_prefill_chunk_host",
     "kvc_prefill_chunk_static", "kvc_status_static", "kvc_prefill_chunk_proxy",
     "kvc_join", "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
-    "kvc_profile_read", "kvc_launch_count", "kvc_last_error",
+    "kvc_profile_read", "kvc_launch_count", "kvc_last_error", "kvc_set_wait_limit", "kvc_selftest_wait_timeout",
 ]
 
 
@@ -69,6 +69,8 @@ def load_library() -> ctypes.CDLL:
     lib.kvc_move_counts.argtypes = [vp, vp, i, ctypes.POINTER(vp)]
     lib.kvc_status.argtypes = [vp, vp, vp]
     lib.kvc_join.argtypes = [vp, vp]
+    lib.kvc_set_wait_limit.argtypes = [vp, ll]
+    lib.kvc_selftest_wait_timeout.argtypes = [vp, vp, vp]
     lib.kvc_kv_bytes.argtypes = [vp, ll, psz, psz, psz]
     lib.kvc_profile_enable.argtypes = [vp, i]
     lib.kvc_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
@@ -162,7 +164,7 @@ class Kvc:
     def reset(self, layer: int = 0, n_layers: Optional[int] = None):
         n_layers = self.cfg.n_layers - layer if n_layers is None else n_layers
         self._check(self._lib.kvc_reset(self._h, layer, n_layers, self.cache[layer].data_ptr(),
-                                        self.blob_bytes, self._stream()))
+                                        self.cache.stride(0), self._stream()))
 
     def prefill_chunk(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, pos0: int,
                       out: Optional[torch.Tensor] = None) -> torch.Tensor:
@@ -195,7 +197,7 @@ class Kvc:
             assert t.stride(-1) == 1 and t.stride(-2) == t.shape[-1] and t.stride(1) == t.shape[-1] * t.shape[-2]
         self._check(self._lib.kvc_prefill_chunk_layers(
             self._h, layer0, nl, _ptr(q), q.stride(0), _ptr(k), _ptr(v), k.stride(0), n, pos0,
-            self.cache[layer0].data_ptr(), self.blob_bytes, self.workspace.data_ptr(), _ptr(out), out.stride(0),
+            self.cache[layer0].data_ptr(), self.cache.stride(0), self.workspace.data_ptr(), _ptr(out), out.stride(0),
             self._stream()))
         return out
 
@@ -272,6 +274,16 @@ class Kvc:
 
     def status(self) -> int:
         return self._lib.kvc_status(self._h, self.workspace.data_ptr(), self._stream())
+
+    def set_wait_limit(self, cycles: int) -> None:
+        self._check(self._lib.kvc_set_wait_limit(self._h, cycles))
+
+    def selftest_wait_timeout(self) -> None:
+        """Enqueues the kernel whose only wait has no producer; ``status()`` then returns KVC_ETIMEOUT."""
+        self._check(self._lib.kvc_selftest_wait_timeout(self._h, self.workspace.data_ptr(), self._stream()))
+
+    def workspace_init(self) -> None:
+        self._check(self._lib.kvc_workspace_init(self._h, self.workspace.data_ptr(), self._stream()))
 
     def kv_bytes(self, seq_len: int) -> Tuple[int, int, int]:
         a, b, c = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()

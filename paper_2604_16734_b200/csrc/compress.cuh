@@ -78,9 +78,9 @@ __device__ __forceinline__ int team_scan_incl(int v, int* scratch, int* total) {
 struct CompressSmem {
   uint64_t q_full, k_full[2], s_full[2], t_free[2];
   uint32_t tmem_base;
-  int abort_flag;
-  float lse2[256];
-  int hist[kSelBins];
+  int wait_ctl[2];           // [0] abort flag, [1] wait limit in units of 1024 cycles (see mbar_wait)
+  alignas(16) float lse2[256];
+  alignas(16) int hist[kSelBins];
   unsigned long long list[2 * (kTeam / 32) + 2];
   int scan_scratch[kTeam / 32 + 1];
   unsigned long long s_prefix;
@@ -112,8 +112,8 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
   int* msrc_g = reinterpret_cast<int*>(slot + p.msrc_off) + static_cast<long long>(g) * p.max_chunk;
   int* mdst_g = reinterpret_cast<int*>(slot + p.mdst_off) + static_cast<long long>(g) * p.max_chunk;
   int* mcount = reinterpret_cast<int*>(slot + p.mcount_off);
-  volatile int* abort_flag = &sh.abort_flag;
-  if (tid == 0) sh.abort_flag = 0;
+  volatile int* abort_flag = sh.wait_ctl;
+  if (tid == 0) { sh.wait_ctl[0] = 0; sh.wait_ctl[1] = p.wait_limit_k; }
   pdl_launch_dependents();                        // the next kernel of the stream may set itself up meanwhile
 
   // ------------------------------------------------------------------------------------ phase 1: scores
@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     }
   } else if constexpr (MODE == kScoreKeyDiff) {
     // Query-agnostic score (Sec. 3.2): anchor mu = mean of the tot keys the cache holds after the append,
-    // score_j = 1 - cos(k_j, mu) for the candidates (>= 0, so its bit pattern orders like an integer; a
+    // score_j = max(0, 1 - cos(k_j, mu)) for the candidates (>= 0, so its bit pattern orders like an integer; a
     // zero key or anchor has cosine 0).  A row is read by lpr lanes of 16 bytes; the CTAs of the cluster
     // take the 128-row tiles round-robin, add their partial sums through distributed shared memory, and
     // every CTA scores its own tiles (second read of K: L2).
@@ -338,8 +338,10 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
             nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
           }
           if (row < r_end && piece == 0) {
+            // fp32 rounding can put the cosine of a key (nearly) parallel to the anchor a little above 1: clamp, so
+            // that the score stays >= 0 and select_key's ordering by bit pattern holds
             const float den = sqrtf(nrm) * mu_norm;
-            score[row] = den > 0.f ? 1.f - dot / den : 1.f;
+            score[row] = den > 0.f ? fmaxf(0.f, 1.f - dot / den) : 1.f;
           }
         }
       }
@@ -526,7 +528,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
       if (sj >= 0) pos[dj] = pos[sj];
     }
   }
-  if (tid == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+  if (tid == 0 && sh.wait_ctl[0]) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
 }
 
 }  // namespace kvc

@@ -23,6 +23,7 @@ struct Geom {
   long long ws_ls;                 // workspace slot stride, bytes (one slot per batched layer)
   int slot0;                       // workspace slot of the call's first layer (0 unless compress runs on the side stream)
   long long lse_off, score_off, msrc_off, mdst_off, mcount_off;   // byte offsets inside a slot
+  int wait_limit_k;                // limit of every device-side wait, in units of 1024 clock cycles
 };
 
 static constexpr int kNumSMs = 148;          // B200

@@ -221,4 +221,23 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
   if (part == 0 && key < p.n_cand) score[key] = acc;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one CTA waits on an mbarrier that nobody will ever arrive on.  With a wait limit
+// of a few thousand cycles the wait gives up, the CTA passes its barrier, records KVC_ETIMEOUT in the status word
+// exactly as the production kernels do, and returns.  Nothing in it can wait longer than the limit.
+// grid 1, block 128.
+__global__ void __launch_bounds__(128) wait_timeout_selftest_kernel(char* __restrict__ ws, int wait_limit_k) {
+  __shared__ uint64_t bar;
+  __shared__ int wait_ctl[2];
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    wait_ctl[0] = 0; wait_ctl[1] = wait_limit_k;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(&bar, 0, wait_ctl);          // phase 0 never completes: returns false after the limit
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || wait_ctl[0])) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+}
+
 }  // namespace kvc

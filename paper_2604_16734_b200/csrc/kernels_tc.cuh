@@ -46,9 +46,11 @@ static constexpr int kStages = 4;                 // K/V ring slots of the atten
 // distributed shared memory: rank s owns rows [s*128/S, (s+1)*128/S) of both tiles, every CTA copies
 // its partial rows (fp32) into the owner's shared memory with remote stores, the cluster
 // synchronises, and each rank combines and writes its rows.  Nothing but the final result goes to HBM.
-// Row tiles per CTA: R = 2 as described, or R = 1 (tile A only; S then alternates between both tiles' TMEM columns):
-// a CTA with one row tile runs its key tiles about 0.7 times as fast per row tile, but exchanges half as much in
-// the combine and doubles the CTA count, which lets a launch that would need S = 4 do with S = 2; the host picks.
+// Row tiles per CTA: R = 2 as described, or R = 1.  A CTA with one row tile runs it twice over: softmax group and
+// issuer t take its key tiles t, t+2, ... with S, P, O, maximum and row sum of their own (tile B's TMEM columns), and
+// the two partial results are merged at the end.  That costs about 1.1 times as much per row tile and key tile, but
+// exchanges half as much in the combine and doubles the CTA count, which lets a launch that would need S = 4 do
+// with S = 2; the host picks.
 // grid (ceil(ceil(n/TOK)/R) * S, Hkv, nl), cluster (S,1,1), block 384,
 // dynamic smem (2 + kStages) * (D/64) * 16 KB + 1 KB.
 static constexpr int kAttnThreads = 384;
@@ -56,8 +58,8 @@ static constexpr int kAttnThreads = 384;
 struct TcSmemAttn {
   uint64_t q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_half[2][2], pv_done[2];
   uint32_t tmem_base;
-  int abort_flag;
-  float stat[2 * 128 * 2];   // key split: (m, l) of the rows this rank owns, [S sources][2 tiles][rows_per][2], S * rows_per = 128
+  int wait_ctl[2];           // [0] abort flag, [1] wait limit in units of 1024 cycles (see mbar_wait)
+  alignas(16) float stat[2 * 128 * 2];   // (read and written as float2) key split: (m, l) of the rows this rank owns, [S sources][2 tiles][rows_per][2], S * rows_per = 128
 };
 
 template <int D>
@@ -106,7 +108,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     }
     // a ring slot is free again once the issuer of every active row tile has committed its MMAs on it
     for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], has_B ? 2 : 1); }
-    sh.abort_flag = 0;
+    sh.wait_ctl[0] = 0; sh.wait_ctl[1] = p.wait_limit_k;
     mbar_fence_init();
   }
   // rows of the Q tiles that TMA never writes (rows >= TOK*G) must still be finite
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sh.tmem_base;
-  volatile int* abort_flag = &sh.abort_flag;
+  volatile int* abort_flag = sh.wait_ctl;
 
   if (warp >= 8) {
     reg_dec<72>();
@@ -633,7 +635,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     tc_fence_after_sync();
     tmem_dealloc(tmem, TMEM_COLS);
   }
-  if (threadIdx.x == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+  if (threadIdx.x == 0 && sh.wait_ctl[0]) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -644,8 +646,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
 struct TcSmemScore {
   uint64_t bar_k, bar_q, bar_s;
   uint32_t tmem_base;
-  int abort_flag;
-  float lse2[256];
+  int wait_ctl[2];           // [0] abort flag, [1] wait limit in units of 1024 cycles (see mbar_wait)
+  alignas(16) float lse2[256];
 };
 
 template <int D>
@@ -669,7 +671,7 @@ __global__ void __launch_bounds__(128) score_tc_kernel(const __grid_constant__ C
 
   if (threadIdx.x == 0) {
     mbar_init(&sh.bar_k, 1); mbar_init(&sh.bar_q, 1); mbar_init(&sh.bar_s, 1);
-    sh.abort_flag = 0;
+    sh.wait_ctl[0] = 0; sh.wait_ctl[1] = p.wait_limit_k;
     mbar_fence_init();
   }
   // observer rows beyond the last group's real rows are padding: keep them finite
@@ -684,7 +686,7 @@ __global__ void __launch_bounds__(128) score_tc_kernel(const __grid_constant__ C
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sh.tmem_base;
-  volatile int* abort_flag = &sh.abort_flag;
+  volatile int* abort_flag = sh.wait_ctl;
   const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
 
   if (threadIdx.x == 0) {
@@ -748,7 +750,7 @@ __global__ void __launch_bounds__(128) score_tc_kernel(const __grid_constant__ C
     tc_fence_after_sync();
     tmem_dealloc(tmem, TMEM_COLS);
   }
-  if (threadIdx.x == 0 && sh.abort_flag) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
+  if (threadIdx.x == 0 && sh.wait_ctl[0]) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
 }
 
 }  // namespace kvc

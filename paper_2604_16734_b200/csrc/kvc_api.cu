@@ -36,6 +36,7 @@ struct kvc_ctx {
   EncodeTiledFn encode;
   bool use_tc;
   bool profiling;
+  int wait_limit_k;              // limit of the kernels' waits, in units of 1024 clock cycles
   struct Prof { int kind; cudaEvent_t a, b; };
   std::vector<Prof> prof;
   // KVC_FLAG_ASYNC_COMPRESS: the side streams, per layer an event after its attention and one after its
@@ -84,7 +85,7 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   if (w > cfg->budget) return KVC_EINVAL;                 // the protected window must fit the budget
   const int G = cfg->n_q_heads / cfg->n_kv_heads;
   if (G > 128) return KVC_EINVAL;
-  if (cfg->device < 0) return KVC_EINVAL;
+  if (cfg->device < 0 || cfg->device >= 64) return KVC_EINVAL;   // per-device tables below hold 64 ordinals
   if ((long long)cfg->budget + cfg->max_chunk > (1ll << 30)) return KVC_EINVAL;
 
   kvc_ctx* c = new (std::nothrow) kvc_ctx();
@@ -115,6 +116,7 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->encode = nullptr;
   c->use_tc = cfg->dtype == KVC_BF16 && !(cfg->flags & KVC_FLAG_CUDA_CORES);
   c->profiling = false;
+  c->wait_limit_k = kvc::kDefaultWaitLimitK;
   for (auto& s : c->side) s = nullptr;
   c->pending.assign(cfg->n_layers, 0);
   c->copy_in = nullptr;
@@ -303,6 +305,26 @@ extern "C" int kvc_move_counts(const kvc_ctx* c, void* workspace, int slot, int*
   return KVC_OK;
 }
 
+extern "C" int kvc_set_wait_limit(kvc_ctx* c, long long cycles) {
+  if (!live(c)) return KVC_ESTATE;
+  if (cycles < 1024 || cycles > (1ll << 40)) return fail(c, KVC_EINVAL, "wait limit %lld outside [1024, 2^40] cycles", cycles);
+  c->wait_limit_k = (int)(cycles >> 10);
+  return KVC_OK;
+}
+
+extern "C" int kvc_selftest_wait_timeout(kvc_ctx* c, void* workspace, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!workspace || !aligned16(workspace)) return fail(c, KVC_EINVAL, "workspace pointer null or misaligned");
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != c->cfg.device)
+    return fail(c, KVC_ESTATE, "current CUDA device %d is not the context's device %d", dev, c->cfg.device);
+  // never more than about 2^21 cycles (a millisecond): the kernel exists to run into its limit
+  const int limit_k = c->wait_limit_k < 2048 ? c->wait_limit_k : 2048;
+  kvc::wait_timeout_selftest_kernel<<<1, 128, 0, (cudaStream_t)stream>>>((char*)workspace, limit_k);
+  c->launches++;
+  return check_cuda(c, cudaGetLastError(), "self-test launch");
+}
+
 extern "C" int kvc_status(kvc_ctx* c, void* workspace, void* stream) {
   if (!live(c)) return KVC_ESTATE;
   if (!workspace) return KVC_EINVAL;
@@ -346,20 +368,27 @@ static int make_map(kvc_ctx* c, CUtensorMap* m, const void* base, const uint64_t
   return KVC_OK;
 }
 
+// cudaFuncSetAttribute acts on the current device only: every kernel that opts into more dynamic shared memory keeps
+// one flag per device ordinal (the caller has checked that the current device is the context's).
+static const int kMaxDevices = 64;
+template <typename Kernel>
+static cudaError_t opt_in_smem(Kernel kernel, int bytes, bool* done_per_device, int dev) {
+  if (done_per_device[dev]) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) done_per_device[dev] = true;
+  return e;
+}
+
 template <typename T, int D>
 static void launch_cc_attn(const Geom& g, const void* q, void* cache, void* out, void* ws, cudaStream_t st) {
   dim3 grid((g.n + 15) / 16, g.Hq, g.nl);
   kvc::attn_cc_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const char*)cache, (T*)out, (char*)ws, g);
 }
 template <typename T, int D>
-static cudaError_t launch_cc_score(const Geom& g, const void* q, void* cache, void* ws, cudaStream_t st) {
+static cudaError_t launch_cc_score(const Geom& g, int dev, const void* q, void* cache, void* ws, cudaStream_t st) {
   const int smem = (kvc::kScoreCcKeys * (D + 4) + 32 * D + 32) * 4;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::score_cc_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool attr_set[kMaxDevices] = {};
+  if (cudaError_t e = opt_in_smem(kvc::score_cc_kernel<T, D>, smem, attr_set, dev)) return e;
   dim3 grid((g.n_cand + kvc::kScoreCcKeys - 1) / kvc::kScoreCcKeys, g.Hkv, g.nl);
   kvc::score_cc_kernel<T, D><<<grid, 128, smem, st>>>((const T*)q, (const char*)cache, (char*)ws, g);
   return cudaSuccess;
@@ -418,16 +447,12 @@ static void attn_launch_shape(const Geom& g, bool allow_split, int* S_out, int* 
 }
 
 template <int D>
-static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+static cudaError_t launch_tc_attn(const Geom& g, int dev, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                   const CUtensorMap& tkin, const CUtensorMap& tvin, void* cache, void* out, void* ws, int S,
                                   int R, bool pdl, cudaStream_t st) {
   const int smem = (2 + kvc::kStages) * (D / 64) * kvc::kSubTileBytes + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool attr_set[kMaxDevices] = {};
+  if (cudaError_t e = opt_in_smem(kvc::attn_tc_kernel<D>, smem, attr_set, dev)) return e;
   const int TOK = 128 / g.G;
   const int groups = ((g.n + TOK - 1) / TOK + R - 1) / R;
   cudaLaunchConfig_t lc;
@@ -444,18 +469,14 @@ static cudaError_t launch_tc_attn(const Geom& g, const CUtensorMap& tq, const CU
 }
 // a2..a4 fused (compress.cuh).  MODE: kvc::kScoresGiven / kScoreAttention / kScoreKeyDiff.
 template <int D, int MODE>
-static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
+static cudaError_t launch_compress(const Geom& g, int dev, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
                                    int elem_bytes, bool pdl, cudaStream_t st) {
   const int score_bytes = MODE == kvc::kScoreAttention ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * kvc::kMaxObsRowsFused * 128 : 0;
   const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4;
   const int smem_min = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
   const int smem_solo = 120 * 1024;                      // more than half an SM: one CTA per SM
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::compress_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_solo);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool attr_set[kMaxDevices] = {};
+  if (cudaError_t e = opt_in_smem(kvc::compress_kernel<D, MODE>, smem_solo, attr_set, dev)) return e;
   // cluster size: spread one kv-head over several SMs when the heads alone cannot fill the GPU
   // (about four key tiles per CTA: below that the two cluster barriers cost more than the tiles)
   const int n_tiles = (g.n_cand + 127) / 128;
@@ -481,15 +502,11 @@ static cudaError_t launch_compress(const Geom& g, const CUtensorMap& tk, const C
 }
 
 template <int D>
-static cudaError_t launch_tc_score(const Geom& g, const CUtensorMap& tk, const CUtensorMap& tqo, void* ws,
+static cudaError_t launch_tc_score(const Geom& g, int dev, const CUtensorMap& tk, const CUtensorMap& tqo, void* ws,
                                    int tok_per_group, cudaStream_t st) {
   const int smem = (D / 64) * (kvc::kSubTileBytes + 256 * 128) + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kvc::score_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool attr_set[kMaxDevices] = {};
+  if (cudaError_t e = opt_in_smem(kvc::score_tc_kernel<D>, smem, attr_set, dev)) return e;
   dim3 grid((g.n_cand + 127) / 128, g.Hkv, g.nl);
   kvc::score_tc_kernel<D><<<grid, 128, smem, st>>>(tk, tqo, (char*)ws, g, tok_per_group);
   return cudaSuccess;
@@ -497,7 +514,8 @@ static cudaError_t launch_tc_score(const Geom& g, const CUtensorMap& tk, const C
 
 static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_ls, const void* k, const void* v,
                      long long kv_ls, int n, long long pos0, void* cache, size_t cache_ls, void* ws, void* out,
-                     long long out_ls, cudaStream_t st, int n_proxy = 0, bool allow_async = true) {
+                     long long out_ls, cudaStream_t st, int n_proxy = 0, bool allow_async = true,
+                     bool clear_status = false) {
   const kvc_config& cf = c->cfg;
   if (layer0 < 0 || nl < 1 || layer0 + nl > cf.n_layers) return fail(c, KVC_EINVAL, "layer range [%d, %d) outside [0, %d)", layer0, layer0 + nl, cf.n_layers);
   if (!q || !k || !v || !cache || !ws || !out) return fail(c, KVC_EINVAL, "null pointer argument");
@@ -552,6 +570,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   g.slot0 = async_compress ? layer0 : 0;
   g.lse_off = c->lse_off; g.score_off = c->score_off; g.msrc_off = c->msrc_off; g.mdst_off = c->mdst_off;
   g.mcount_off = c->mcount_off;
+  g.wait_limit_k = c->wait_limit_k;
   const bool evict = g.tot > g.B;                      // Alg. 1: "if |C| > M"
   const bool f32 = cf.dtype == KVC_F32;
   const int D = cf.head_dim;
@@ -590,6 +609,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   const bool pdl = pdl_main;
   cudaError_t e = cudaSuccess;
   if (int rc = wait_pending(c, layer0, layer0 + nl, st)) return rc;    // a compress kernel of an earlier block may still run
+  // every host check has passed: from here on work is enqueued.  A workspace that keeps an earlier user's contents
+  // (the built-in scratch array) gets its status word cleared first.
+  if (clear_status)
+    if (int rc = check_cuda(c, cudaMemsetAsync(ws, 0, kvc::kWsHeaderBytes, st), "cudaMemsetAsync(status word)")) return rc;
   // a0 append (the tensor-core attention kernel appends by itself)
   if (!c->use_tc) {
     ProfScope ps(c, 0, st);
@@ -610,8 +633,8 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   if (c->use_tc) {
     int S = 1, R = 2;
     attn_launch_shape(g, !(cf.flags & 4u), &S, &R);
-    e = D == 128 ? launch_tc_attn<128>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st)
-                 : launch_tc_attn<64>(g, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st);
+    e = D == 128 ? launch_tc_attn<128>(g, dev, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st)
+                 : launch_tc_attn<64>(g, dev, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st);
   } else if (f32) {
     if (D == 128) launch_cc_attn<float, 128>(g, q, cache, out, ws, st); else launch_cc_attn<float, 64>(g, q, cache, out, ws, st);
   } else {
@@ -635,11 +658,11 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
       // fusing up to 256 rows was measured and is slower, the stand-alone kernel spreads the key tiles wider)
       ProfScope ps(c, 2, st);
       if (c->use_tc) {
-        e = D == 128 ? launch_tc_score<128>(g, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, tk, tqo, ws, tok_per_group, st);
+        e = D == 128 ? launch_tc_score<128>(g, dev, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, dev, tk, tqo, ws, tok_per_group, st);
       } else if (f32) {
-        e = D == 128 ? launch_cc_score<float, 128>(g, q, cache, ws, st) : launch_cc_score<float, 64>(g, q, cache, ws, st);
+        e = D == 128 ? launch_cc_score<float, 128>(g, dev, q, cache, ws, st) : launch_cc_score<float, 64>(g, dev, q, cache, ws, st);
       } else {
-        e = D == 128 ? launch_cc_score<__nv_bfloat16, 128>(g, q, cache, ws, st) : launch_cc_score<__nv_bfloat16, 64>(g, q, cache, ws, st);
+        e = D == 128 ? launch_cc_score<__nv_bfloat16, 128>(g, dev, q, cache, ws, st) : launch_cc_score<__nv_bfloat16, 64>(g, dev, q, cache, ws, st);
       }
       if (e != cudaSuccess) return check_cuda(c, e, "score launch");
       c->launches++;
@@ -647,10 +670,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     // (a2 +) a3 select + a4 compact
     {
       ProfScope ps(c, 3, st);
-      if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, tk, tk, cache, ws, (int)c->elem, pdl, st);
-      else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st)
-                                         : launch_compress<64, kvc::kScoreAttention>(g, tk, tqo, cache, ws, (int)c->elem, pdl, st);
-      else e = launch_compress<64, kvc::kScoresGiven>(g, tk, tk, cache, ws, (int)c->elem, pdl, st);
+      if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, st);
+      else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, st)
+                                         : launch_compress<64, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, st);
+      else e = launch_compress<64, kvc::kScoresGiven>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, st);
     }
     if (e != cudaSuccess) return check_cuda(c, e, "compress launch");
     c->launches++;
@@ -757,7 +780,6 @@ extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host,
 // In host code `g_static_ws` is only a handle for the runtime, not a device address; the address
 // each device gives it is looked up once per device and cached here.
 static __device__ __align__(256) unsigned char g_static_ws[KVC_STATIC_WS_BYTES];
-static const int kMaxDevices = 64;
 static void* g_static_ws_ptr[kMaxDevices] = {nullptr};
 
 static int static_ws_for_current_device(kvc_ctx* c, void** ptr) {
@@ -787,10 +809,9 @@ extern "C" int kvc_prefill_chunk_static(kvc_ctx* c, int layer, const void* q, co
   void* ws = nullptr;
   int rc = static_ws_for_current_device(c, &ws);
   if (rc) return rc;
-  // the array keeps the previous call's contents: only the status word has to start at zero
-  rc = check_cuda(c, cudaMemsetAsync(ws, 0, kvc::kWsHeaderBytes, (cudaStream_t)stream), "cudaMemsetAsync(static scratch)");
-  if (rc) return rc;
-  return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, ws, out, 0, (cudaStream_t)stream, 0, false);
+  // the array keeps the previous call's contents: only the status word has to start at zero, and it is cleared
+  // once the argument and state checks have passed (a rejected call enqueues nothing)
+  return run_chunk(c, layer, 1, q, 0, k, v, 0, n, pos0, cache, 0, ws, out, 0, (cudaStream_t)stream, 0, false, true);
 }
 
 extern "C" int kvc_status_static(kvc_ctx* c, void* stream) {

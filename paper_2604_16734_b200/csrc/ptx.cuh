@@ -6,9 +6,10 @@
 
 namespace kvc {
 
-// Every device-side wait is bounded: after this many clock cycles a waiter gives up, records
-// KVC_ETIMEOUT in the status word and the kernel drains and exits normally.
-static constexpr long long kWaitLimitCycles = 2000000000LL;   // about one second
+// Every device-side wait is bounded: after the context's wait limit (about one second of clock cycles unless the
+// host sets another, counted in units of 1024 cycles) a waiter gives up, records KVC_ETIMEOUT in the status word
+// and the kernel drains and exits normally.
+static constexpr int kDefaultWaitLimitK = 1953125;   // x 1024 cycles: about one second
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -39,16 +40,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  `abort_flag` is a shared-memory word: once any waiter times out it is set and every
-// later wait returns false immediately, so the whole CTA falls through to its exit path.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait.  `wait_ctl` points at two shared-memory words: [0] the abort flag -- once any waiter times out it
+// is set and every later wait returns false immediately, so the whole CTA falls through to its exit path -- and
+// [1] the wait limit in units of 1024 clock cycles (read only on the slow path).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* wait_ctl) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
+    if (wait_ctl[0]) return false;
+    if (((clock64() - t0) >> 10) > static_cast<long long>(wait_ctl[1])) {
+      wait_ctl[0] = 1;
       return false;
     }
   }

@@ -10,7 +10,7 @@ from paper_2604_16734_b200.binding import (Kvc, KvcError, KVC_FLAG_CUDA_CORES, K
                                            KVC_ESTATE)
 from paper_2604_16734_b200.workloads import CONFIGS, Workload, reduced
 
-from parity_util import compare_chunk, make_oracle, run_workload_parity
+from parity_util import assert_output_bound, compare_chunk, make_oracle, run_workload_parity
 
 pytestmark = pytest.mark.gpu
 
@@ -44,7 +44,7 @@ def test_c2_llava_shaped_two_layers(flags):
     cfg = reduced(CONFIGS["C2"], n_layers=2)
     kvc = _kvc_for(cfg, flags)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0, 1]), [0, 1])
-    assert worst["err_out"] <= 2e-2
+    assert_output_bound(worst, torch.bfloat16)
 
 
 @pytest.mark.parametrize("flags", [0, KVC_FLAG_CUDA_CORES])
@@ -52,14 +52,14 @@ def test_c3_tiled_group_of_seven(flags):
     cfg = reduced(CONFIGS["C3"], n_layers=1, n_units=2)       # 2 tiles of 576 + 128 text, B = 1024, G = 7
     kvc = _kvc_for(cfg, flags)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0])
-    assert worst["err_out"] <= 2e-2
+    assert_output_bound(worst, torch.bfloat16)
 
 
 def test_c4_video_frames():
     cfg = reduced(CONFIGS["C4"], n_layers=1, n_units=12)      # 12 frames of 196 -> 2352 > B = 2048
     kvc = _kvc_for(cfg)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0])
-    assert worst["err_out"] <= 2e-2
+    assert_output_bound(worst, torch.bfloat16)
     kvc.reset()
     run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], teacher_forced=True)
 
@@ -68,7 +68,7 @@ def test_c5_long_video_blocks():
     cfg = reduced(CONFIGS["C5"], n_layers=1, n_units=36)      # 5184 vision tokens -> 6 blocks, B = 4096
     kvc = _kvc_for(cfg)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=[0, 7])
-    assert worst["err_out"] <= 2e-2
+    assert_output_bound(worst, torch.bfloat16)
 
 
 # ------------------------------------------------------------------------------------------------
@@ -81,7 +81,7 @@ def test_full_size_one_layer(name, kv_heads, flags):
     cfg = reduced(CONFIGS[name], n_layers=1)
     kvc = _kvc_for(cfg, flags)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=kv_heads)
-    assert worst["err_out"] <= 2e-2
+    assert_output_bound(worst, torch.bfloat16)
     # the cache never exceeds the budget, and ends exactly at it once the prefix is longer than B
     K, V, pos, ln = kvc.cache_view(0)
     assert ln == min(cfg.n_tokens, cfg.budget)
@@ -99,7 +99,7 @@ def test_query_agnostic_policy(name, units, kv_heads):
     cfg = reduced(CONFIGS[name], n_layers=1, n_units=units)
     kvc = _kvc_for(cfg, policy=binding.KVC_SCORE_KEYDIFF)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=kv_heads, policy="keydiff")
-    assert worst["err_out"] <= (1e-4 if cfg.dtype == "fp32" else 2e-2)
+    assert_output_bound(worst, cfg.torch_dtype)
     assert kvc.cache_view(0)[3] == min(cfg.n_tokens, cfg.budget)
 
 
@@ -128,7 +128,7 @@ def test_hybrid_bulk_first_block(name, units, kv_heads):
     assert sched[0] == (0, cfg.budget) and sched[0][1] > cfg.chunk
     kvc = _kvc_for(cfg)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=kv_heads, chunks=sched)
-    assert worst["err_out"] <= (1e-4 if cfg.dtype == "fp32" else 2e-2)
+    assert_output_bound(worst, cfg.torch_dtype)
     assert kvc.cache_view(0)[3] == cfg.budget
     # the exception is for an empty cache only
     q, k, v = _layers(cfg, [0])[0]
@@ -179,7 +179,7 @@ def test_block_size_study_workload(block):
     cfg = reduced(CONFIGS["T4"], n_layers=1, n_units=4).scaled(chunk=block)     # 3136 vision tokens > B = 2048
     kvc = _kvc_for(cfg)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0]), [0], kv_heads=[1])
-    assert worst["err_out"] <= 2e-2
+    assert_output_bound(worst, torch.bfloat16)
     logical, physical, full = kvc.kv_bytes(cfg.n_tokens)
     assert logical == 2 * 4 * 128 * 2 * 2048 and physical >= 2 * 4 * 128 * 2 * (2048 + block)   # the bound grows with the block
 
@@ -304,6 +304,14 @@ def test_duplicate_keys_tie_break_keeps_older():
     assert ln == 8 and kept == list(range(len(kept)))       # identical scores: the older entries stay
 
 
+def _same_to_bf16_rounding(a, b):
+    """Two bf16 results of sums taken in different orders: equal within 2e-2, or at most one bf16 ulp apart."""
+    a, b = a.float(), b.float()
+    diff = (a - b).abs()
+    ulp = torch.exp2(torch.floor(torch.log2(torch.maximum(a.abs(), b.abs()).clamp_min(2.0 ** -126))) - 7)
+    return bool(((diff <= 2e-2) | (diff <= ulp)).all())
+
+
 def test_layer_batched_call_matches_per_layer_calls():
     cfg = reduced(CONFIGS["C4"], n_layers=3, n_units=11)
     wl = Workload(cfg)
@@ -321,13 +329,80 @@ def test_layer_batched_call_matches_per_layer_calls():
     assert a.status() == 0 and b.status() == 0
     # the key range is split over more CTAs when fewer layers share a launch, so the two paths sum in a
     # different order: outputs agree to bf16 rounding, not bit for bit
-    # (two bf16 roundings of nearly the same number may land one ulp apart: 2^-7 relative)
-    diff = (out_a.float() - out_b.float()).abs() / (out_a.float().abs() / 2).clamp_min(1.0)
-    assert diff.max().item() <= 2e-2
+    assert _same_to_bf16_rounding(out_a, out_b)
     for l in range(3):
         Ka, Va, Pa, la = a.cache_view(l); Kb, Vb, Pb, lb = b.cache_view(l)
         assert la == lb == cfg.budget
         assert torch.equal(Pa[:, :la], Pb[:, :lb]) and torch.equal(Ka[:, :la], Kb[:, :lb]) and torch.equal(Va[:, :la], Vb[:, :lb])
+
+
+@pytest.mark.parametrize("name,units,samples", [("C4", None, [(0, 1), (17, 6), (31, 3)]), ("C5", 43, [(5, 0), (30, 7)])])
+def test_layer_batched_at_full_depth(name, units, samples):
+    # The layer-batched entry point with ALL layers of the configuration in one launch, as `bench.py --mode batched`
+    # uses it: 256 (kv-head, layer) pairs, so the compress kernel runs two CTAs per SM with the small shared-memory
+    # request and the attention kernel runs in several waves.  Checked two ways: against one-layer-per-call runs of
+    # the same blocks (caches bit-exact, outputs to bf16 rounding) and against the oracle on sampled (layer, kv-head)
+    # pairs, block by block.  C4: the whole prefix.  C5: the first blocks up to three past the budget.
+    from parity_util import pre_state
+    full = CONFIGS[name]
+    cfg = reduced(full, n_layers=full.n_layers, n_units=units)
+    L = cfg.n_layers
+    wl = Workload(cfg, device="cuda")
+    Q = torch.empty(L, cfg.n_tokens, cfg.n_q_heads, cfg.head_dim, dtype=torch.bfloat16, device="cuda")
+    K = torch.empty(L, cfg.n_tokens, cfg.n_kv_heads, cfg.head_dim, dtype=torch.bfloat16, device="cuda")
+    V = torch.empty_like(K)
+    for l in range(L):
+        Q[l], K[l], V[l] = wl.layer(l)
+    del wl
+    a = _kvc_for(cfg); b = _kvc_for(cfg)
+    from parity_util import install_guards, check_guards
+    install_guards(b)
+    orc = make_oracle(cfg)
+    layers = sorted({l for l, _ in samples})
+    heads = {l: sorted(g for ll, g in samples if ll == l) for l in layers}
+    out_a = torch.empty(L, cfg.chunk, cfg.n_q_heads, cfg.head_dim, dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty_like(out_a)
+    worst = dict(err_out=0.0, ulp_escapes=0)
+    for pos0, n in cfg.chunks():
+        for l in range(L):
+            a.prefill_chunk(l, Q[l, pos0:pos0 + n], K[l, pos0:pos0 + n], V[l, pos0:pos0 + n], pos0, out_a[l, :n])
+        pre = {l: pre_state(b, l) for l in range(L)}
+        b.prefill_chunk_layers(0, Q[:, pos0:pos0 + n], K[:, pos0:pos0 + n], V[:, pos0:pos0 + n], pos0, out_b[:, :n])
+        torch.cuda.synchronize()
+        assert a.status() == 0 and b.status() == 0
+        check_guards(b)
+        assert _same_to_bf16_rounding(out_a[:, :n], out_b[:, :n])
+        for l in layers:
+            st = compare_chunk(b, orc, l, Q[l, pos0:pos0 + n].cpu(), K[l, pos0:pos0 + n].cpu(), V[l, pos0:pos0 + n].cpu(), pos0,
+                               kv_heads=heads[l], out_gpu=out_b[l, :n], slot=l, pre=pre[l])
+            worst["err_out"] = max(worst["err_out"], st["err_out"]); worst["ulp_escapes"] += st["ulp_escapes"]
+        for l in range(L):
+            Ka, Va, Pa, la = a.cache_view(l); Kb, Vb, Pb, lb = b.cache_view(l)
+            assert la == lb
+            if torch.equal(Pa[:, :la], Pb[:, :lb]):
+                assert torch.equal(Ka[:, :la], Kb[:, :lb]) and torch.equal(Va[:, :la], Vb[:, :lb])
+                continue
+            # The two paths split the key range differently, so their log-sum-exps, and with them the scores, differ
+            # in the last bits: over the ~10^4 selections of this run a few cut-offs fall between two candidates
+            # whose scores are that close, and the paths may then keep different ones.  Accept exactly that: every
+            # entry kept by only one path scores within 1e-5 (relative) of the others; then let path a continue
+            # from path b's cache.
+            pos_before, len_before = pre[l]
+            _, score_b = b.workspace_view(l)
+            for g in range(cfg.n_kv_heads):
+                sa, sb = set(Pa[g, :la].tolist()), set(Pb[g, :lb].tolist())
+                if sa == sb:
+                    continue
+                phys = np.concatenate([pos_before[g], pos0 + np.arange(n)])
+                sc = dict(zip(phys.tolist(), score_b[g, :len(phys)].double().cpu().tolist()))
+                disputed = [sc[x] for x in (sa ^ sb)]
+                assert len(sa) == len(sb) and max(disputed) - min(disputed) <= 1e-5 * max(disputed), (l, g, sorted(sa ^ sb), disputed)
+                worst["near_ties"] = worst.get("near_ties", 0) + 1
+            a.cache[l].copy_(b.cache[l])
+    print(f"layer-batched {name} at full depth: {worst}")
+    assert worst.get("near_ties", 0) <= 8
+    assert_output_bound(worst, torch.bfloat16)
+    assert b.cache_view(0)[3] == min(cfg.budget, cfg.n_tokens)
 
 
 @pytest.mark.parametrize("name,units,n_layers,graph", [("C2", None, 4, False), ("C2", None, 4, True),
@@ -380,7 +455,7 @@ def test_compress_on_side_stream_against_the_oracle_two_layers():
     cfg = reduced(CONFIGS["C4"], n_layers=2, n_units=9)
     kvc = _kvc_for(cfg, KVC_FLAG_ASYNC_COMPRESS)
     worst = run_workload_parity(kvc, cfg, _layers(cfg, [0, 1]), [0, 1], kv_heads=[2, 7])
-    assert worst["err_out"] <= 2e-2
+    assert_output_bound(worst, torch.bfloat16)
 
 
 def test_cuda_graph_replay_matches_direct_calls():

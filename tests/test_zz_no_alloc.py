@@ -35,6 +35,20 @@ def test_static_scratch_matches_workspace_entry_point(dtype, hq, hkv, d):
         tol = 1e-4 if dtype == torch.float32 else 2e-2
         assert (out_ref.float() - out_sta.float()).abs().max().item() <= tol
         p += n
+    # a warm call allocates nothing: the free device memory is the same before and after it (inputs made up front)
+    n = 40
+    q = torch.randn(n, hq, d, device="cuda").to(dtype)
+    k = torch.randn(n, hkv, d, device="cuda").to(dtype)
+    v = torch.randn(n, hkv, d, device="cuda").to(dtype)
+    out = torch.empty_like(q)
+    out_ref = ref.prefill_chunk(0, q, k, v, p)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    sta.prefill_chunk_static(0, q, k, v, p, out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert sta.status_static() == 0
+    assert (out_ref.float() - out.float()).abs().max().item() <= tol
     Kr, Vr, Pr, lr = ref.cache_view(0)
     Ks, Vs, Ps, ls = sta.cache_view(0)
     assert lr == ls == budget
@@ -49,3 +63,18 @@ def test_static_scratch_rejects_oversized_configuration():
     with pytest.raises(KvcError) as e:
         big.prefill_chunk_static(0, x, x, x, 0)
     assert e.value.code == KVC_EINVAL and "scratch" in str(e.value)
+
+
+def test_static_scratch_rejected_call_enqueues_nothing():
+    # a call that fails its argument checks launches nothing (the clear of the shared status word included:
+    # it is enqueued only after the checks) and leaves the context usable
+    kvc = Kvc(1, 4, 2, 128, torch.bfloat16, 64, 32)
+    x = torch.zeros(8, 4, 128, device="cuda", dtype=torch.bfloat16); y = torch.zeros(8, 2, 128, device="cuda", dtype=torch.bfloat16)
+    kvc.prefill_chunk_static(0, x, y, y, 0)
+    assert kvc.status_static() == 0
+    before = kvc.launch_count()
+    big = torch.zeros(40, 4, 128, device="cuda", dtype=torch.bfloat16); bigk = torch.zeros(40, 2, 128, device="cuda", dtype=torch.bfloat16)
+    with pytest.raises(KvcError) as e:
+        kvc.prefill_chunk_static(0, big, bigk, bigk, 8)            # n > max_chunk
+    assert e.value.code == KVC_EINVAL
+    assert kvc.launch_count() == before and kvc.status_static() == 0

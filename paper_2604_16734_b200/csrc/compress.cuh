@@ -30,6 +30,7 @@ namespace kvc {
 static constexpr int kCompressThreads = 512;
 static constexpr int kDigitBits = 11;
 static constexpr int kSelBins = 1 << kDigitBits;
+static constexpr int kRankMax = 256;          // keys of the cut-off bin that are ranked directly instead of by further rounds
 static constexpr int kMaxKeysSmem = 6144;     // candidates whose keys fit the shared-memory table (48 KB)
 static constexpr int kMaxMovesSmem = 2048;    // moves whose (src, dst) fit the shared-memory tables (16 KB)
 static constexpr int kMaxObsRowsFused = 128;  // observer rows (w * G) the fused scoring phase takes
@@ -41,50 +42,20 @@ __device__ __forceinline__ unsigned long long select_key(float score, int pos) {
          static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(pos));
 }
 
-// The selection and the listing run on a team of kTeam threads: the whole block (measured: a quarter of
-// it pays less per barrier but more per key, and loses).
+// The selection and the listing run on the whole block (measured: a quarter of it pays less per barrier but more
+// per key, and loses).
 static constexpr int kTeam = kCompressThreads;
-__device__ __forceinline__ void team_sync() { named_barrier(3, kTeam); }
-
-// Inclusive scan of one int per team thread; returns the inclusive value and the team total.
-// scratch: kTeam / 32 + 1 ints of shared memory.  Only warp 0 combines the warp totals: a value that
-// every thread reads costs one load per warp, so 16 such values would cost 256 loads.
-__device__ __forceinline__ int team_scan_incl(int v, int* scratch, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
-  }
-  team_sync();                            // scratch may still be read from a previous scan
-  if (lane == 31) scratch[warp] = incl;
-  team_sync();
-  if (warp == 0) {
-    int t = lane < kTeam / 32 ? scratch[lane] : 0, ti = t;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, ti, o);
-      if (lane >= o) ti += y;
-    }
-    if (lane < kTeam / 32) scratch[lane] = ti - t;   // exclusive warp offsets
-    if (lane == 31) scratch[kTeam / 32] = ti;
-  }
-  team_sync();
-  *total = scratch[kTeam / 32];
-  return incl + scratch[warp];
-}
 
 struct CompressSmem {
   uint64_t q_full, k_full[2], s_full[2], t_free[2];
   uint32_t tmem_base;
   int wait_ctl[2];           // [0] abort flag, [1] wait limit in units of 1024 cycles (see mbar_wait)
   alignas(16) float lse2[256];
-  alignas(16) int hist[kSelBins];
+  alignas(16) int hist[2][kSelBins];    // histograms of two consecutive rounds (the second doubles as the list of the last bin's keys)
   unsigned long long list[2 * (kTeam / 32) + 2];
   int scan_scratch[kTeam / 32 + 1];
   unsigned long long s_prefix;
-  int s_remaining, s_bin_count;
+  int s_remaining, s_bin_count, s_count;
 };
 
 // grid (Cn, Hkv, nl), cluster (Cn,1,1), block 512.
@@ -363,75 +334,115 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
   int* tab_src = reinterpret_cast<int*>(smem + kMaxKeysSmem * 8);                    // 8 KB
   int* tab_dst = tab_src + kMaxMovesSmem;                                            // 8 KB
   const bool keys_in_smem = p.n_cand <= kMaxKeysSmem;
-  if (keys_in_smem)
-    for (int j = tid; j < p.n_cand; j += kCompressThreads) keys[j] = select_key(__ldcg(score + j), pos[j]);
-  __syncthreads();
   auto key_of = [&](int j) -> unsigned long long {
     return keys_in_smem ? keys[j] : select_key(__ldcg(score + j), pos[j]);
   };
-
-  if (p.n_keep > 0) {
-    {                                                            // (all kTeam threads)
-      // The bits above the highest bit in which any two keys differ are common to all keys (scores of
-      // similar magnitude share their exponent bits): start the descent below them, so that the first
-      // digit already spreads the keys over many bins instead of piling them onto a few counters.
-      unsigned long long k_and = ~0ull, k_or = 0ull;
-      for (int j = tid; j < p.n_cand; j += kTeam) { const unsigned long long k = key_of(j); k_and &= k; k_or |= k; }
-      unsigned a_lo = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(k_and)), a_hi = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(k_and >> 32));
-      unsigned o_lo = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or)), o_hi = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or >> 32));
-      if (lane == 0) { sh.list[warp] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[kTeam / 32 + warp] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
-      team_sync();
-      if (warp == 0) {                                           // one warp folds the 32 partial results
-        const unsigned long long pa = lane < kTeam / 32 ? sh.list[lane] : ~0ull, po = lane < kTeam / 32 ? sh.list[kTeam / 32 + lane] : 0ull;
-        a_lo = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(pa)); a_hi = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(pa >> 32));
-        o_lo = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(po)); o_hi = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(po >> 32));
-        if (lane == 0) { sh.list[2 * (kTeam / 32)] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[2 * (kTeam / 32) + 1] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
-      }
-      team_sync();
-      k_and = sh.list[2 * (kTeam / 32)]; k_or = sh.list[2 * (kTeam / 32) + 1];
-      const unsigned long long differ = k_and ^ k_or;           // != 0: at least two distinct keys (n_cand > n_keep >= 1)
-      const int top = 63 - __clzll(static_cast<long long>(differ));
-      int shift = top >= kDigitBits - 1 ? top - (kDigitBits - 1) : 0, bits = top - shift + 1;
-      team_sync();                                               // sh.list is reused below
-      if (tid == 0) { sh.s_prefix = top == 63 ? 0ull : (k_or >> (top + 1)) << (top + 1); sh.s_remaining = p.n_keep; }
-      while (true) {
-        for (int i = tid; i < kSelBins; i += kTeam) sh.hist[i] = 0;
-        team_sync();
-        const unsigned long long prefix = sh.s_prefix;
-        const int remaining = sh.s_remaining;
-        const int hi = shift + bits;         // bits [hi, 64) are already decided
-        for (int j = tid; j < p.n_cand; j += kTeam) {
-          const unsigned long long key = key_of(j);
-          if (hi >= 64 || (key >> hi) == (prefix >> hi)) atomicAdd(&sh.hist[(key >> shift) & ((1u << bits) - 1)], 1);
-        }
-        team_sync();
-        // descending scan: thread t owns the BPT bins from kSelBins - 1 - BPT*t downwards
-        constexpr int BPT = kSelBins / kTeam;
-        const int b0 = kSelBins - 1 - BPT * tid;
-        int mine = 0;
+  // One pass builds the keys (four independent loads in flight per thread: the scores come from L2), folds the
+  // AND and the OR of all keys -- the bits above the highest bit in which any two keys differ are common to all of
+  // them (scores of similar magnitude share their exponent bits), and the descent starts below them, so that the
+  // first digit already spreads the keys over many bins -- and clears the first histogram.
+  unsigned long long k_and = ~0ull, k_or = 0ull;
+  for (int j0 = tid; j0 < p.n_cand; j0 += 4 * kCompressThreads) {
+    float sc[4];
+    int ps[4];
 #pragma unroll
-        for (int i = 0; i < BPT; ++i) mine += sh.hist[b0 - i];
-        int total;
-        const int incl = team_scan_incl(mine, sh.scan_scratch, &total);
-        int excl = incl - mine;
-        if (excl < remaining && remaining <= incl) {             // the cut-off lies in one of my bins
-          int b = b0, h = sh.hist[b0];
-          while (excl + h < remaining) { excl += h; --b; h = sh.hist[b]; }
-          sh.s_prefix = prefix | (static_cast<unsigned long long>(b) << shift);
-          sh.s_remaining = remaining - excl;                     // rank inside the chosen bin, 1-based
-          sh.s_bin_count = h;
-        }
-        team_sync();
-        // Done when every bit is decided, or when the whole bin survives (its rank equals its size): then
-        // the prefix with zeros below it separates the retained keys from the others.
-        if (shift == 0 || sh.s_remaining == sh.s_bin_count) break;
-        bits = shift >= kDigitBits ? kDigitBits : shift;
-        shift -= bits;
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + u * kCompressThreads;
+      if (j < p.n_cand) { sc[u] = __ldcg(score + j); ps[u] = pos[j]; }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + u * kCompressThreads;
+      if (j < p.n_cand) {
+        const unsigned long long k = select_key(sc[u], ps[u]);
+        if (keys_in_smem) keys[j] = k;
+        k_and &= k; k_or |= k;
       }
     }
-    __syncthreads();
   }
-  const unsigned long long thr = p.n_keep > 0 ? sh.s_prefix : ~0ull;   // n_keep == 0: nothing among the candidates survives
+  {
+    const unsigned a_lo = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(k_and)), a_hi = __reduce_and_sync(0xffffffffu, static_cast<unsigned>(k_and >> 32));
+    const unsigned o_lo = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or)), o_hi = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or >> 32));
+    if (lane == 0) { sh.list[warp] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[kTeam / 32 + warp] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
+  }
+  for (int i = tid; i < kSelBins; i += kTeam) sh.hist[0][i] = 0;
+  __syncthreads();
+  unsigned long long thr = ~0ull;                                // n_keep == 0: nothing among the candidates survives
+  if (p.n_keep > 0) {
+    k_and = ~0ull; k_or = 0ull;
+#pragma unroll
+    for (int w2 = 0; w2 < kTeam / 32; ++w2) { k_and &= sh.list[w2]; k_or |= sh.list[kTeam / 32 + w2]; }   // (every thread: the same values)
+    const unsigned long long differ = k_and ^ k_or;             // != 0: at least two distinct keys (n_cand > n_keep >= 1)
+    const int top = 63 - __clzll(static_cast<long long>(differ));
+    int shift = top >= kDigitBits - 1 ? top - (kDigitBits - 1) : 0, bits = top - shift + 1;
+    // state of the descent, the same in every thread: the bits decided so far and the rank (1-based, from the top) of
+    // the cut-off among the keys that share them
+    unsigned long long prefix = top == 63 ? 0ull : (k_or >> (top + 1)) << (top + 1);
+    int remaining = p.n_keep, hb = 0;
+    while (true) {
+      int* hist = sh.hist[hb];
+      const int hi = shift + bits;           // bits [hi, 64) are already decided
+      for (int j = tid; j < p.n_cand; j += kTeam) {
+        const unsigned long long key = key_of(j);
+        if (hi >= 64 || (key >> hi) == (prefix >> hi)) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1)], 1);
+      }
+      for (int i = tid; i < kSelBins; i += kTeam) sh.hist[hb ^ 1][i] = 0;   // for the next round
+      __syncthreads();
+      // descending scan: thread t owns the BPT bins from kSelBins - 1 - BPT*t downwards; scan inside the warp by
+      // shuffles, across the warps by reading the totals of the warps before (one barrier)
+      constexpr int BPT = kSelBins / kTeam;
+      const int b0 = kSelBins - 1 - BPT * tid;
+      int mine = 0;
+#pragma unroll
+      for (int i = 0; i < BPT; ++i) mine += hist[b0 - i];
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      if (lane == 31) sh.scan_scratch[warp] = incl;
+      __syncthreads();
+      for (int w2 = 0; w2 < warp; ++w2) incl += sh.scan_scratch[w2];
+      int excl = incl - mine;
+      if (excl < remaining && remaining <= incl) {               // the cut-off lies in one of my bins
+        int b = b0, h = hist[b0];
+        while (excl + h < remaining) { excl += h; --b; h = hist[b]; }
+        sh.s_prefix = prefix | (static_cast<unsigned long long>(b) << shift);
+        sh.s_remaining = remaining - excl;                       // rank inside the chosen bin, 1-based
+        sh.s_bin_count = h;
+        sh.s_count = 0;
+      }
+      __syncthreads();
+      prefix = sh.s_prefix; remaining = sh.s_remaining;
+      const int h = sh.s_bin_count;
+      // Done when every bit is decided, or when the whole bin survives (its rank equals its size): then
+      // the prefix with zeros below it separates the retained keys from the others.
+      if (shift == 0 || remaining == h) { thr = prefix; break; }
+      if (h <= kRankMax) {
+        // few keys left in the cut-off bin: list them and rank them directly (keys are unique: exactly one of them
+        // has `remaining - 1` larger ones) instead of descending further
+        unsigned long long* lst = reinterpret_cast<unsigned long long*>(sh.hist[hb ^ 1]);
+        for (int j = tid; j < p.n_cand; j += kTeam) {
+          const unsigned long long key = key_of(j);
+          if ((key >> shift) == (prefix >> shift)) lst[atomicAdd(&sh.s_count, 1)] = key;
+        }
+        __syncthreads();
+        if (tid < h) {
+          const unsigned long long my = lst[tid];
+          int larger = 0;
+          for (int i = 0; i < h; ++i) larger += lst[i] > my;
+          if (larger == remaining - 1) sh.s_prefix = my;
+        }
+        __syncthreads();
+        thr = sh.s_prefix;
+        break;
+      }
+      bits = shift >= kDigitBits ? kDigitBits : shift;
+      shift -= bits;
+      hb ^= 1;
+    }
+  }
 
   // ------------------------------------------------------------------------------------ phase 3: compaction
   // holes: evicted entries in rows [0, B); survivors: retained entries in rows [B, tot), both in ascending
@@ -457,19 +468,14 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
       holes += __popc(__ballot_sync(0xffffffffu, valid && j < n_lo && !keep));
       surv += __popc(__ballot_sync(0xffffffffu, valid && j >= n_lo && keep));
     }
-    // both counts share one scan when they fit 16 bits each (tot < 65536); lane 0 carries the warp's counts
-    int total_holes, off_h, off_s;
-    if (p.tot < 65536) {
-      int total;
-      const int mine = lane == 0 ? (holes | (surv << 16)) : 0;
-      const int packed = team_scan_incl(mine, sh.scan_scratch, &total);
-      off_h = __shfl_sync(0xffffffffu, (packed & 0xffff) - holes, 0);
-      off_s = __shfl_sync(0xffffffffu, (packed >> 16) - surv, 0);
-      total_holes = total & 0xffff;
-    } else {
-      int total_surv;
-      off_h = __shfl_sync(0xffffffffu, team_scan_incl(lane == 0 ? holes : 0, sh.scan_scratch, &total_holes) - holes, 0);
-      off_s = __shfl_sync(0xffffffffu, team_scan_incl(lane == 0 ? surv : 0, sh.scan_scratch, &total_surv) - surv, 0);
+    // offsets of the warp's holes and survivors: the counts of the warps before it (one barrier)
+    if (lane == 0) { sh.scan_scratch[warp] = holes; sh.list[warp] = static_cast<unsigned long long>(surv); }
+    __syncthreads();
+    int total_holes = 0, off_h = 0, off_s = 0;
+    for (int w2 = 0; w2 < kTeam / 32; ++w2) {
+      const int hw = sh.scan_scratch[w2];
+      if (w2 < warp) { off_h += hw; off_s += static_cast<int>(sh.list[w2]); }
+      total_holes += hw;
     }
     for (int base = s0; base < s1; base += 32) {
       const int j = base + lane;

@@ -57,6 +57,7 @@ static constexpr int kAttnThreads = 384;
 
 struct TcSmemAttn {
   uint64_t q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_half[2][2], pv_done[2];
+  uint64_t comb_full;        // key split: the other ranks' partial rows have landed in this CTA's shared memory
   uint32_t tmem_base;
   int wait_ctl[2];           // [0] abort flag, [1] wait limit in units of 1024 cycles (see mbar_wait)
   alignas(16) float stat[2 * 128 * 2];   // (read and written as float2) key split: (m, l) of the rows this rank owns, [S sources][2 tiles][rows_per][2], S * rows_per = 128
@@ -109,6 +110,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     // a ring slot is free again once the issuer of every active row tile has committed its MMAs on it
     for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], has_B ? 2 : 1); }
     sh.wait_ctl[0] = 0; sh.wait_ctl[1] = p.wait_limit_k;
+    mbar_init(&sh.comb_full, 1);
+    // key split with one row tile: every other rank of the cluster will copy its partial of this rank's rows here
+    if (S > 1 && !has_B) mbar_expect_tx(&sh.comb_full, (S - 1) * (128 / S) * D * 4);
     mbar_fence_init();
   }
   // rows of the Q tiles that TMA never writes (rows >= TOK*G) must still be finite
@@ -276,9 +280,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       }
     }
     __syncwarp();
-    if (S > 1) {                                             // the two cluster barriers of the combine below
+    if (S > 1) {                                             // the cluster barriers of the combine below
       cluster_arrive(); cluster_wait();
       cluster_arrive(); cluster_wait();
+      if (!has_B) { cluster_arrive(); cluster_wait(); }
     }
   } else {
     reg_inc<216>();
@@ -560,8 +565,28 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             if (owner != split) stat_addr = dsmem_addr(stat_addr, owner);
             dsmem_st_v2(stat_addr, (have && l > 0.f) ? m_ref : -INFINITY, have ? l : 0.f);
           }
+          const bool bulk = !has_B;                             // (uniform over the cluster: its CTAs share the row tiles)
+          if (bulk) fence_proxy_async_smem();                   // the rows just written are read by bulk copies
           named_barrier(1, nthr);                               // the staging tile is complete
           constexpr int CPR = D / 4;                            // 16-byte chunks per row
+          if (bulk) {
+            // One row tile: the rows of every other owner leave in ONE bulk copy each (shared memory to the owner's
+            // shared memory, completing on the owner's barrier; this GPU's own memory, no multicast); only this
+            // rank's own rows are copied by the threads.  Per-thread remote stores moved 13 B/clk.
+            if (threadIdx.x == 0) {
+              for (int owner = 0; owner < S; ++owner) {
+                if (owner == split) continue;
+                bulk_copy_to_cluster(dsmem_addr(smem_u32(stage + (split * 2 + tt) * rows_per * D), owner),
+                                     smem_u32(stg + owner * rows_per * D), rows_per * D * 4,
+                                     dsmem_addr(smem_u32(&sh.comb_full), owner));
+              }
+            }
+            for (int idx = threadIdx.x; idx < rows_per * CPR; idx += nthr) {
+              const int lr = idx / CPR, chunk = idx % CPR;
+              *reinterpret_cast<uint4*>(stage + ((split * 2 + tt) * rows_per + lr) * D + chunk * 4) =
+                  *reinterpret_cast<const uint4*>(stg + (split * rows_per + lr) * D + chunk * 4);
+            }
+          } else {
 #pragma unroll 4
           for (int idx = threadIdx.x; idx < 128 * CPR; idx += nthr) {
             const int row = idx / CPR, chunk = idx % CPR;
@@ -571,11 +596,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             if (owner != split) dst = dsmem_addr(dst, owner);
             dsmem_st_v4_b32(dst, v4.x, v4.y, v4.z, v4.w);
           }
+          }
           named_barrier(1, nthr);                               // the staging tile may be overwritten
         }
       }
-      cluster_arrive();                                         // all partials have landed; no remote access after this
-      cluster_wait();
+      cluster_arrive();                                         // all partials have landed (bulk copies: see below); no
+      cluster_wait();                                           // remote access is started after this
+      // the bulk copies of the other ranks complete on this CTA's barrier, not at the cluster barrier
+      if (!has_B) ok = mbar_wait(&sh.comb_full, 0, abort_flag) && ok;
       {
         const int r0 = min(128, split * rows_per), nrows = min(128, r0 + rows_per) - r0;
         const int per_tile = nrows * (D / 32);                  // work items: (row, group of 32 columns)
@@ -626,6 +654,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           }
         }
       }
+      // A CTA must not exit while a bulk copy still reads its staging tile: every rank has waited for the copies
+      // addressed to it, so once all of them are here every copy is complete.
+      if (!has_B) { cluster_arrive(); cluster_wait(); }
     }
   }
 

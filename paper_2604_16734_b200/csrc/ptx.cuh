@@ -260,6 +260,12 @@ __device__ __forceinline__ void dsmem_st_v4_b32(uint32_t addr, uint32_t a, uint3
 __device__ __forceinline__ void dsmem_st_v2(uint32_t addr, float a, float b) {
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the same cluster (addresses from
+// dsmem_addr); its bytes are counted on an mbarrier of the destination CTA.  Addresses and size: multiples of 16.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(bar_cluster) : "memory");
+}
 __device__ __forceinline__ float dsmem_ld_f32(uint32_t addr) {
   float v;
   asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");

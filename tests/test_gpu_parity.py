@@ -538,3 +538,20 @@ def test_kv_bytes_stay_at_the_budget_bound():
     logical, physical, full = kvc.kv_bytes(cfg.n_tokens)
     assert physical <= kvc.blob_bytes * 2 and logical < physical < full
     assert kvc.cache.numel() == 2 * kvc.blob_bytes          # nothing else is ever allocated for the cache
+
+
+@pytest.mark.parametrize("dtype,policy", [(torch.bfloat16, "attn"), (torch.float32, "attn"), (torch.bfloat16, "keydiff")])
+def test_budget_beyond_the_shared_memory_tables(dtype, policy):
+    # more candidates than the selection keeps in shared memory (6144) and more moves than its move tables hold
+    # (2048): the keys are then re-read from the workspace and the move lists go through global memory
+    from oracle.kvc_oracle import KVCOracle
+    hq = hkv = 1; d = 64
+    B, c, w = 7000, 2300, 16
+    kvc = Kvc(1, hq, hkv, d, dtype, B, c, w, policy=binding.KVC_SCORE_KEYDIFF if policy == "keydiff" else 0)
+    orc = KVCOracle(1, hq, hkv, d, B, w, policy=policy)
+    torch.manual_seed(77)
+    p = 0
+    for n in (B, 2300, 2200):
+        q = torch.randn(n, hq, d).to(dtype); k = (torch.randn(n, hkv, d) + 0.3).to(dtype); v = torch.randn(n, hkv, d).to(dtype)
+        compare_chunk(kvc, orc, 0, q, k, v, p)
+        p += n

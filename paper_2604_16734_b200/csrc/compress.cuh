@@ -20,6 +20,7 @@
 // keys share and stops as soon as the bin that holds the cut-off survives as a whole.
 #pragma once
 #include <cuda.h>
+#include <type_traits>
 #include "geom.cuh"
 #include "ptx.cuh"
 
@@ -51,7 +52,6 @@ struct CompressSmem {
   uint32_t tmem_base;
   int wait_ctl[2];           // [0] abort flag, [1] wait limit in units of 1024 cycles (see mbar_wait)
   alignas(16) float lse2[256];
-  alignas(16) int hist[2][kSelBins];    // histograms of two consecutive rounds (the second doubles as the list of the last bin's keys)
   unsigned long long list[2 * (kTeam / 32) + 2];
   int scan_scratch[kTeam / 32 + 1];
   unsigned long long s_prefix;
@@ -60,7 +60,7 @@ struct CompressSmem {
 
 // grid (Cn, Hkv, nl), cluster (Cn,1,1), block 512.
 // dynamic smem: the larger of the scoring buffers (two K tiles + up to 128 observer rows) and of the key
-// and move tables (64 KB), + 1 KB.
+// and move tables with the two histograms (80 KB), + 1 KB.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __grid_constant__ CUtensorMap tm_k,
                                                                        const __grid_constant__ CUtensorMap tm_qobs,
@@ -333,10 +333,9 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);           // 48 KB
   int* tab_src = reinterpret_cast<int*>(smem + kMaxKeysSmem * 8);                    // 8 KB
   int* tab_dst = tab_src + kMaxMovesSmem;                                            // 8 KB
+  // histograms of two consecutive rounds (the second doubles as the list of the last bin's keys): 2 x 8 KB
+  int (*hists)[kSelBins] = reinterpret_cast<int (*)[kSelBins]>(smem + kMaxKeysSmem * 8 + 2 * kMaxMovesSmem * 4);
   const bool keys_in_smem = p.n_cand <= kMaxKeysSmem;
-  auto key_of = [&](int j) -> unsigned long long {
-    return keys_in_smem ? keys[j] : select_key(__ldcg(score + j), pos[j]);
-  };
   // One pass builds the keys (four independent loads in flight per thread: the scores come from L2), folds the
   // AND and the OR of all keys -- the bits above the highest bit in which any two keys differ are common to all of
   // them (scores of similar magnitude share their exponent bits), and the descent starts below them, so that the
@@ -365,8 +364,21 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     const unsigned o_lo = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or)), o_hi = __reduce_or_sync(0xffffffffu, static_cast<unsigned>(k_or >> 32));
     if (lane == 0) { sh.list[warp] = (static_cast<unsigned long long>(a_hi) << 32) | a_lo; sh.list[kTeam / 32 + warp] = (static_cast<unsigned long long>(o_hi) << 32) | o_lo; }
   }
-  for (int i = tid; i < kSelBins; i += kTeam) sh.hist[0][i] = 0;
+  for (int i = tid; i < kSelBins; i += kTeam) hists[0][i] = 0;
   __syncthreads();
+  // Selection and listing exist twice, for keys in shared memory and for keys re-read from the workspace: with the
+  // choice made per access the compiler issues the global loads of the second form in both cases.
+  const int n_lo = min(p.B, p.tot);
+  const int max_moves = min(p.n, p.tot - p.B);                   // at most this many entries sit at or above row B
+  const bool tabs_in_smem = max_moves <= kMaxMovesSmem;
+  int* msrc = tabs_in_smem ? tab_src : msrc_g;                   // with global tables every CTA writes all entries
+  int* mdst = tabs_in_smem ? tab_dst : mdst_g;                   // itself (same values) and reads only its own writes
+  auto select_and_list = [&](auto in_smem) {
+  constexpr bool kInSmem = decltype(in_smem)::value;
+  auto key_of = [&](int j) -> unsigned long long {
+    if constexpr (kInSmem) return keys[j];
+    else return select_key(__ldcg(score + j), pos[j]);
+  };
   unsigned long long thr = ~0ull;                                // n_keep == 0: nothing among the candidates survives
   if (p.n_keep > 0) {
     k_and = ~0ull; k_or = 0ull;
@@ -380,13 +392,13 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     unsigned long long prefix = top == 63 ? 0ull : (k_or >> (top + 1)) << (top + 1);
     int remaining = p.n_keep, hb = 0;
     while (true) {
-      int* hist = sh.hist[hb];
+      int* hist = hists[hb];
       const int hi = shift + bits;           // bits [hi, 64) are already decided
       for (int j = tid; j < p.n_cand; j += kTeam) {
         const unsigned long long key = key_of(j);
         if (hi >= 64 || (key >> hi) == (prefix >> hi)) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1)], 1);
       }
-      for (int i = tid; i < kSelBins; i += kTeam) sh.hist[hb ^ 1][i] = 0;   // for the next round
+      for (int i = tid; i < kSelBins; i += kTeam) hists[hb ^ 1][i] = 0;   // for the next round
       __syncthreads();
       // descending scan: thread t owns the BPT bins from kSelBins - 1 - BPT*t downwards; scan inside the warp by
       // shuffles, across the warps by reading the totals of the warps before (one barrier)
@@ -422,7 +434,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
       if (h <= kRankMax) {
         // few keys left in the cut-off bin: list them and rank them directly (keys are unique: exactly one of them
         // has `remaining - 1` larger ones) instead of descending further
-        unsigned long long* lst = reinterpret_cast<unsigned long long*>(sh.hist[hb ^ 1]);
+        unsigned long long* lst = reinterpret_cast<unsigned long long*>(hists[hb ^ 1]);
         for (int j = tid; j < p.n_cand; j += kTeam) {
           const unsigned long long key = key_of(j);
           if ((key >> shift) == (prefix >> shift)) lst[atomicAdd(&sh.s_count, 1)] = key;
@@ -447,50 +459,45 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
   // ------------------------------------------------------------------------------------ phase 3: compaction
   // holes: evicted entries in rows [0, B); survivors: retained entries in rows [B, tot), both in ascending
   // row order.  Entry j is retained iff it is protected (j >= n_cand) or its key >= thr.
-  const int n_lo = min(p.B, p.tot);
-  const int max_moves = min(p.n, p.tot - p.B);                   // at most this many entries sit at or above row B
-  const bool tabs_in_smem = max_moves <= kMaxMovesSmem;
-  int* msrc = tabs_in_smem ? tab_src : msrc_g;                   // with global tables every CTA writes all entries
-  int* mdst = tabs_in_smem ? tab_dst : mdst_g;                   // itself (same values) and reads only its own writes
   {
-    // Each warp owns a contiguous segment of the rows, walked 32 rows at a time (lane = row, so the
-    // shared-memory keys are read without bank conflicts).  Pass 1 counts the warp's holes (rows below
-    // B) and survivors (rows from B on), one scan over the warps turns the counts into offsets,
-    // pass 2 writes the row indices in ascending order.
-    const int seg = ((p.tot + kTeam / 32 - 1) / (kTeam / 32) + 31) & ~31;   // rows per warp, a multiple of 32
-    const int s0 = warp * seg, s1 = min(s0 + seg, p.tot);
+    // Every thread owns a run of consecutive rows: it counts its holes (rows below B) and survivors (rows from B
+    // on), one scan over the block (shuffles inside the warps, one barrier across them) turns the counts into
+    // offsets, and a second walk over the same rows writes the row indices, in ascending order.
+    const int rpt = (p.tot + kTeam - 1) / kTeam;                 // rows per thread
+    const int r0 = min(tid * rpt, p.tot), r1 = min(r0 + rpt, p.tot);
     auto retained = [&](int j) { return j >= p.n_cand || key_of(j) >= thr; };
-    int holes = 0, surv = 0;
-    for (int base = s0; base < s1; base += 32) {
-      const int j = base + lane;
-      const bool valid = j < s1;
-      const bool keep = valid && retained(j);
-      holes += __popc(__ballot_sync(0xffffffffu, valid && j < n_lo && !keep));
-      surv += __popc(__ballot_sync(0xffffffffu, valid && j >= n_lo && keep));
+    unsigned long long mine = 0;                                  // holes in the low word, survivors in the high word
+    for (int j = r0; j < r1; ++j) {
+      const bool keep = retained(j);
+      if (j < n_lo) mine += keep ? 0ull : 1ull;
+      else mine += keep ? (1ull << 32) : 0ull;
     }
-    // offsets of the warp's holes and survivors: the counts of the warps before it (one barrier)
-    if (lane == 0) { sh.scan_scratch[warp] = holes; sh.list[warp] = static_cast<unsigned long long>(surv); }
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) sh.list[warp] = incl;
     __syncthreads();
-    int total_holes = 0, off_h = 0, off_s = 0;
+    unsigned long long before = 0, all = 0;
     for (int w2 = 0; w2 < kTeam / 32; ++w2) {
-      const int hw = sh.scan_scratch[w2];
-      if (w2 < warp) { off_h += hw; off_s += static_cast<int>(sh.list[w2]); }
-      total_holes += hw;
+      const unsigned long long tw = sh.list[w2];
+      if (w2 < warp) before += tw;
+      all += tw;
     }
-    for (int base = s0; base < s1; base += 32) {
-      const int j = base + lane;
-      const bool valid = j < s1;
-      const bool keep = valid && retained(j);
-      const bool is_hole = valid && j < n_lo && !keep, is_surv = valid && j >= n_lo && keep;
-      const unsigned mh = __ballot_sync(0xffffffffu, is_hole), ms = __ballot_sync(0xffffffffu, is_surv);
-      const unsigned below = (1u << lane) - 1;
-      if (is_hole) mdst[off_h + __popc(mh & below)] = j;
-      if (is_surv) msrc[off_s + __popc(ms & below)] = j;
-      off_h += __popc(mh);
-      off_s += __popc(ms);
+    const unsigned long long excl = before + incl - mine;
+    int off_h = static_cast<int>(excl & 0xffffffffu), off_s = static_cast<int>(excl >> 32);
+    const int total_holes = static_cast<int>(all & 0xffffffffu);
+    for (int j = r0; j < r1; ++j) {
+      const bool keep = retained(j);
+      if (j < n_lo) { if (!keep) mdst[off_h++] = j; }
+      else if (keep) msrc[off_s++] = j;
     }
     if (tid == 0) sh.s_remaining = total_holes;                  // == number of survivors: the cache returns to B
   }
+  };
+  if (keys_in_smem) select_and_list(std::true_type{}); else select_and_list(std::false_type{});
   __syncthreads();
   const int total_holes = sh.s_remaining;
   if (rank == 0 && tid == 0) mcount[g] = total_holes;

@@ -472,17 +472,16 @@ template <int D, int MODE>
 static cudaError_t launch_compress(const Geom& g, int dev, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
                                    int elem_bytes, bool pdl, cudaStream_t st) {
   const int score_bytes = MODE == kvc::kScoreAttention ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * kvc::kMaxObsRowsFused * 128 : 0;
-  const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4;
+  const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4 + 2 * kvc::kSelBins * 4;   // keys, move tables, histograms
   const int smem_min = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
   const int smem_solo = 120 * 1024;                      // more than half an SM: one CTA per SM
   static bool attr_set[kMaxDevices] = {};
   if (cudaError_t e = opt_in_smem(kvc::compress_kernel<D, MODE>, smem_solo, attr_set, dev)) return e;
   // cluster size: spread one kv-head over several SMs when the heads alone cannot fill the GPU
-  // (about four key tiles per CTA: below that the two cluster barriers cost more than the tiles)
   const int n_tiles = (g.n_cand + 127) / 128;
   int Cn = (int)(kvc::kNumSMs / ((long long)g.Hkv * g.nl));
-  if (Cn > 8) Cn = 8;
-  const int tiles_per_cta = MODE == kvc::kScoreKeyDiff ? 2 : 4;   // the CUDA-core score reads every tile twice: spread it wider
+  if (Cn > 8) Cn = 8;                                     // portable cluster size limit
+  const int tiles_per_cta = 2;                            // fewer, and the cluster barriers cost more than the tiles
   if (Cn > (n_tiles + tiles_per_cta - 1) / tiles_per_cta) Cn = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
   if (Cn < 1) Cn = 1;
   // Two CTAs share an SM only when there are more CTAs than SMs (then one scores while the other selects);

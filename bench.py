@@ -396,9 +396,12 @@ def time_steps(fn, steps, barrier):
     return e0.elapsed_time(e1) / 1e3, t0, t1
 
 
-def profile_pass(r: Runner, steps: int, batched: bool = False):
-    """Per-kernel CUDA-event durations (on the launching stream) and exact algorithmic work: one call per
-    (block, layer), or with `batched` one call per block with the layer index in the launch grid."""
+def profile_pass(r: Runner, steps: int, batched: bool = False, events: bool = False):
+    """Per-kernel durations and exact algorithmic work: one call per (block, layer), in stream order, or with
+    `batched` one call per block with the layer index in the launch grid.  The durations are device-side time
+    stamps taken inside the kernels (global timer; per launch from the earliest begin of work, past the wait for
+    the preceding kernel, to the latest end over its CTAs): no event pair sits between consecutive launches, so
+    they overlap as they do in the timed step, and the sum of the durations fits inside the step."""
     saved = (r.kvc, r.flags)
     r.kvc, r.flags = r.kvc_in_order, r.flags & ~16
     kv, cfg = r.kvc, r.cfg
@@ -422,12 +425,25 @@ def profile_pass(r: Runner, steps: int, batched: bool = False):
                 work[s]["bytes"] += wv["bytes"]; work[s]["flops"] += wv["flops"]
         n_c = min(n_c + n - t, cfg.budget)
     torch.cuda.synchronize()
-    kv.profile_enable(True)
+    per_step = kv.launch_count()
+    (r.step_batched if batched else r.step_direct)()
+    torch.cuda.synchronize()
+    per_step = kv.launch_count() - per_step
+    kv.profile_device(per_step * steps + 16)
     for _ in range(steps):
         (r.step_batched if batched else r.step_direct)()
-    torch.cuda.synchronize()
-    ms, cnt = kv.profile_read()
-    kv.profile_enable(False)
+    ms, cnt, span_ms = kv.profile_device_read()
+    kv.profile_device(0)
+    # the same launches bracketed by CUDA events on the launching stream (a pair per launch: each kernel alone on the
+    # GPU, launch latency and the events themselves included)
+    ev_ms = ev_cnt = None
+    if events:
+        kv.profile_enable(True)
+        for _ in range(min(steps, 3)):
+            (r.step_batched if batched else r.step_direct)()
+        torch.cuda.synchronize()
+        ev_ms, ev_cnt = kv.profile_read()
+        kv.profile_enable(False)
     r.kvc, r.flags = saved
     per = {}
     for s in STEPS:
@@ -435,6 +451,8 @@ def profile_pass(r: Runner, steps: int, batched: bool = False):
             per[s] = dict(ms_total_per_step=ms[s] / steps, launches_per_step=cnt[s] // steps,
                           us_per_launch=1e3 * ms[s] / cnt[s], bytes_per_step=work[s]["bytes"],
                           flops_per_step=work[s]["flops"])
+            if ev_cnt and ev_cnt[s]:
+                per[s]["us_per_launch_cuda_events"] = 1e3 * ev_ms[s] / ev_cnt[s]
     return per
 
 
@@ -531,36 +549,46 @@ def measure(cfg, args, L, local_rank, rank, world, dist, barrier, peaks, steps, 
     # ---- per-kernel durations and rooflines (rank 0, outside the timed region)
     per, per_b, roof = {}, {}, None
     if rank == 0 and not args.no_profile:
-        per = rates(profile_pass(r, max(3, min(steps, 10)) if primary else 3), peaks)
+        per = rates(profile_pass(r, max(3, min(steps, 10)) if primary else 3, events=True), peaks)
         ridge = peaks["tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
         dom = max(per, key=lambda s: per[s]["ms_total_per_step"])
         d = per[dom]
         ai = d["flops_per_step"] / max(d["bytes_per_step"], 1)
+        # `achieved` rests on CUDA events around every launch of the kernel (the slower, self-contained figure: launch
+        # latency and the events are inside it); the device-stamped duration, which is what the launch occupies in the
+        # in-order step, is given beside it
+        ev_sec = d.get("us_per_launch_cuda_events", d["us_per_launch"]) * 1e-6 * d["launches_per_step"]
+        ev_tflops, ev_gbs = d["flops_per_step"] / ev_sec / 1e12, d["bytes_per_step"] / ev_sec / 1e9
         if cfg.dtype == "bf16" and dom == "attention" and ai > ridge:
             # the kernel is timed inside a long step: the sustained peak is its denominator; the burst figure beside it
-            roof = dict(kernel=dom, bound="tensor", achieved=d["tflops"], peak=peaks["tflops_sustained"], unit="TFLOP/s",
-                        frac=d["tflops"] / peaks["tflops_sustained"], traffic=None,
+            roof = dict(kernel=dom, bound="tensor", achieved=ev_tflops, peak=peaks["tflops_sustained"], unit="TFLOP/s",
+                        frac=ev_tflops / peaks["tflops_sustained"], traffic=None,
                         peak_source=peaks["source"] + " (sustained bf16)", peak_burst=peaks["tflops_burst"],
-                        frac_of_burst_peak=d["tflops"] / peaks["tflops_burst"])
+                        frac_of_burst_peak=ev_tflops / peaks["tflops_burst"],
+                        achieved_device_stamps=d["tflops"], frac_device_stamps=d["tflops"] / peaks["tflops_sustained"],
+                        frac_of_burst_peak_device_stamps=d["tflops"] / peaks["tflops_burst"])
         else:
-            roof = dict(kernel=dom, bound="hbm", achieved=d["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=d["gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"])
+            roof = dict(kernel=dom, bound="hbm", achieved=ev_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=ev_gbs / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"],
+                        achieved_device_stamps=d["gbs"], frac_device_stamps=d["gbs"] / peaks["hbm_gbs"])
         roof["traffic"] = ncu_traffic(cfg.name, dom) if L == cfg.n_layers else None
         roof["algorithmic_bytes_per_launch"] = d["bytes_per_step"] / max(d["launches_per_step"], 1)
         roof["algorithmic_flops_per_launch"] = d["flops_per_step"] / max(d["launches_per_step"], 1)
-        roof["us_per_launch"] = d["us_per_launch"]
+        roof["us_per_launch"] = d.get("us_per_launch_cuda_events", d["us_per_launch"])
+        roof["us_per_launch_device_stamps"] = d["us_per_launch"]
         roof["arithmetic_intensity"] = ai
-        roof["timing"] = "CUDA events around every launch on the launching stream, every kernel alone on the GPU"
-        # the kernels' event-timed durations against the step they have to fit into
+        roof["timing"] = ("achieved / frac: CUDA events around every launch on the launching stream, kernels in stream order; "
+                          "*_device_stamps: time stamps inside the kernel (global timer, earliest begin of work, past the wait "
+                          "for the preceding kernel, to the latest end over the CTAs of a launch)")
+        # the kernels' durations against the step they have to fit into
         kernel_ms_sum = sum(x["ms_total_per_step"] for x in per.values())
         out["kernel_ms_sum"] = kernel_ms_sum
         out["overlap"] = dict(
             ms_per_step_in_order=in_order_ms, ms_per_step=ms_per_step,
             hidden_by_side_streams_ms=(in_order_ms - ms_per_step) if in_order_ms is not None else None,
             kernel_ms_sum_over_in_order=kernel_ms_sum / in_order_ms if in_order_ms else None,
-            note="kernel_ms_sum brackets every launch with an event pair (a few us each, no overlap between "
-                 "consecutive launches); in the in-order step consecutive launches overlap through programmatic "
-                 "dependent launch")
+            note="kernel_ms_sum adds the device-stamped durations of all launches of an in-order step; what the in-order "
+                 "step holds beyond it is the time between launches (launch latency, cache resets)")
         out["roofline_step"] = step_roofline(cfg, per, L, ms_per_step, peaks)
         if in_order_ms is not None and out["roofline_step"]:
             out["roofline_step"]["frac_in_order"] = out["roofline_step"]["bound_ms"] / in_order_ms

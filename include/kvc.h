@@ -253,6 +253,17 @@ int kvc_kv_bytes(const kvc_ctx* ctx, long long seq_len, size_t* logical, size_t*
 int kvc_profile_enable(kvc_ctx* ctx, int on);
 int kvc_profile_read(kvc_ctx* ctx, double* ms, long long* launches);
 
+/* Per-kernel timing without events, for launches of a few microseconds (an event pair costs as much and keeps
+ * consecutive launches from overlapping).  After kvc_profile_device(ctx, records, capacity, stream) -- records:
+ * DEVICE, capacity x 16 bytes, 16-byte aligned, cleared by the call on `stream` -- every kernel of the context's later
+ * calls stamps the nanosecond global timer when a CTA begins its work (past the wait for the preceding kernel) and
+ * when it ends, and the launch's record keeps the earliest begin and the latest end; launches beyond `capacity` are
+ * not recorded.  records = NULL switches it off.  kvc_profile_device_read takes a HOST copy of the records (made by
+ * the caller after synchronising) and ADDS, per kernel index as in kvc_profile_read, the durations in milliseconds
+ * and the launch counts; *span_ms (may be NULL) receives the time from the first begin to the last end. */
+int kvc_profile_device(kvc_ctx* ctx, void* records, long long capacity, void* stream);
+int kvc_profile_device_read(kvc_ctx* ctx, const void* records_host, double* ms, long long* launches, double* span_ms);
+
 /* Number of kernel launches the library has enqueued through this context so far. */
 long long kvc_launch_count(const kvc_ctx* ctx);
 

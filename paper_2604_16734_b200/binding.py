@@ -26,6 +26,7 @@ EXPORTS = [
     "kvc_prefill_chunk_static", "kvc_status_static", "kvc_prefill_chunk_proxy",
     "kvc_join", "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
     "kvc_profile_read", "kvc_launch_count", "kvc_last_error", "kvc_set_wait_limit", "kvc_selftest_wait_timeout",
+    "kvc_profile_device", "kvc_profile_device_read",
 ]
 
 
@@ -74,6 +75,8 @@ def load_library() -> ctypes.CDLL:
     lib.kvc_kv_bytes.argtypes = [vp, ll, psz, psz, psz]
     lib.kvc_profile_enable.argtypes = [vp, i]
     lib.kvc_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
+    lib.kvc_profile_device.argtypes = [vp, vp, ll, vp]
+    lib.kvc_profile_device_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll), ctypes.POINTER(ctypes.c_double)]
     lib.kvc_launch_count.argtypes = [vp]
     lib.kvc_launch_count.restype = ll
     lib.kvc_last_error.argtypes = [vp]
@@ -300,6 +303,26 @@ class Kvc:
         self._check(self._lib.kvc_profile_read(self._h, ms, cnt))
         names = ("append", "attention", "score", "compress", "unused")
         return dict(zip(names, list(ms))), dict(zip(names, list(cnt)))
+
+    def profile_device(self, capacity: int) -> None:
+        """Starts device-side time stamps for the next ``capacity`` launches (0 stops them)."""
+        if capacity <= 0:
+            self._stamps = None
+            self._check(self._lib.kvc_profile_device(self._h, None, 0, self._stream()))
+            return
+        self._stamps = torch.empty(capacity * 2, dtype=torch.int64, device=self.device)
+        self._check(self._lib.kvc_profile_device(self._h, self._stamps.data_ptr(), capacity, self._stream()))
+
+    def profile_device_read(self):
+        """({step: milliseconds}, {step: launches}, span in ms) of the launches stamped since profile_device()."""
+        torch.cuda.synchronize(self.device)
+        host = self._stamps.cpu()
+        ms = (ctypes.c_double * 5)()
+        cnt = (ctypes.c_longlong * 5)()
+        span = ctypes.c_double()
+        self._check(self._lib.kvc_profile_device_read(self._h, host.data_ptr(), ms, cnt, ctypes.byref(span)))
+        names = ("append", "attention", "score", "compress", "unused")
+        return dict(zip(names, list(ms))), dict(zip(names, list(cnt))), span.value
 
     def launch_count(self) -> int:
         return self._lib.kvc_launch_count(self._h)

@@ -115,6 +115,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
       if (lane == 0) {
         tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_qobs);
         pdl_wait();
+        stamp_begin(p);
         bool ok = true;
         if (my_tiles > 0) {
           mbar_expect_tx(&sh.q_full, NSUB * p.w * p.G * 128);
@@ -209,6 +210,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     float* s_sum = s_part + (kCompressThreads / 32) * 128;         // [d] this CTA's sum (read by the cluster)
     float* s_mu = s_sum + 128;                                      // [d] the anchor, [d] = its norm
     pdl_wait();
+    if (tid == 0) stamp_begin(p);
     const int d = p.d, epl = 16 / elem_bytes;                       // elements per 16-byte piece: 8 (bf16) or 4 (fp32)
     const int lpr = d / epl, rpw = 32 / lpr;                        // lanes per row, rows per warp and step
     const int sub = lane / lpr, piece = lane % lpr;
@@ -319,7 +321,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     }
     __syncthreads();
   } else {
-    if (tid == 0) pdl_wait();
+    if (tid == 0) { pdl_wait(); stamp_begin(p); }
     __syncthreads();
   }
   if (Cn > 1) {                                       // every score of this kv-head is in the workspace
@@ -541,6 +543,8 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
       if (sj >= 0) pos[dj] = pos[sj];
     }
   }
+  __syncthreads();
+  if (tid == 0) stamp_end(p);
   if (tid == 0 && sh.wait_ctl[0]) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
 }
 

@@ -24,10 +24,23 @@ struct Geom {
   int slot0;                       // workspace slot of the call's first layer (0 unless compress runs on the side stream)
   long long lse_off, score_off, msrc_off, mdst_off, mcount_off;   // byte offsets inside a slot
   int wait_limit_k;                // limit of every device-side wait, in units of 1024 clock cycles
+  // measurement runs only (else null): this launch's pair of time stamps, {earliest begin of work, latest end} over
+  // its CTAs, in nanoseconds of the global timer
+  unsigned long long* stamps;
 };
 
 static constexpr int kNumSMs = 148;          // B200
 static constexpr int kWsHeaderBytes = 256;   // status word lives at byte 0 of the workspace
+
+// Device-side duration of a launch: a CTA stamps the begin of its work once it is past the wait for the preceding
+// kernel, and its end when it is done; the launch's record keeps the minimum and the maximum.
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void stamp_begin(const Geom& p) { if (p.stamps) atomicMin(p.stamps, global_timer_ns()); }
+__device__ __forceinline__ void stamp_end(const Geom& p) { if (p.stamps) atomicMax(p.stamps + 1, global_timer_ns()); }
 
 __device__ __forceinline__ char* ws_slot(char* ws, const Geom& p, int slot) {
   return ws + kWsHeaderBytes + static_cast<long long>(p.slot0 + slot) * p.ws_ls;

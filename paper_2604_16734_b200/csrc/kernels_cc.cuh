@@ -15,23 +15,27 @@ __global__ void __launch_bounds__(256) append_kernel(const T* __restrict__ k, co
                                                      char* __restrict__ cache, Geom p) {
   pdl_launch_dependents();                 // the attention kernel may set itself up meanwhile
   pdl_wait();                              // the previous block's compaction still reads and writes this cache
+  if (threadIdx.x == 0) stamp_begin(p);
   const int layer = blockIdx.z;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (row >= p.n * p.Hkv) return;
-  const int t = row / p.Hkv, g = row % p.Hkv;
-  char* blob = cache + layer * p.cache_ls;
-  const int vec_per_row = p.d * (int)sizeof(T) / 16;
-  const uint4* ksrc = reinterpret_cast<const uint4*>(k + layer * p.kv_ls + (static_cast<long long>(t) * p.Hkv + g) * p.d);
-  const uint4* vsrc = reinterpret_cast<const uint4*>(v + layer * p.kv_ls + (static_cast<long long>(t) * p.Hkv + g) * p.d);
-  const long long dst_row = static_cast<long long>(g) * p.cap + p.n_c + t;
-  uint4* kdst = reinterpret_cast<uint4*>(blob + dst_row * p.d * sizeof(T));
-  uint4* vdst = reinterpret_cast<uint4*>(blob + p.v_off + dst_row * p.d * sizeof(T));
-  for (int i = lane; i < vec_per_row; i += 32) {
-    kdst[i] = ksrc[i];
-    vdst[i] = vsrc[i];
+  if (row < p.n * p.Hkv) {
+    const int t = row / p.Hkv, g = row % p.Hkv;
+    char* blob = cache + layer * p.cache_ls;
+    const int vec_per_row = p.d * (int)sizeof(T) / 16;
+    const uint4* ksrc = reinterpret_cast<const uint4*>(k + layer * p.kv_ls + (static_cast<long long>(t) * p.Hkv + g) * p.d);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(v + layer * p.kv_ls + (static_cast<long long>(t) * p.Hkv + g) * p.d);
+    const long long dst_row = static_cast<long long>(g) * p.cap + p.n_c + t;
+    uint4* kdst = reinterpret_cast<uint4*>(blob + dst_row * p.d * sizeof(T));
+    uint4* vdst = reinterpret_cast<uint4*>(blob + p.v_off + dst_row * p.d * sizeof(T));
+    for (int i = lane; i < vec_per_row; i += 32) {
+      kdst[i] = ksrc[i];
+      vdst[i] = vsrc[i];
+    }
+    if (lane == 0) reinterpret_cast<int*>(blob + p.pos_off)[dst_row] = static_cast<int>(p.pos0 + t);
   }
-  if (lane == 0) reinterpret_cast<int*>(blob + p.pos_off)[dst_row] = static_cast<int>(p.pos0 + t);
+  __syncthreads();
+  if (threadIdx.x == 0) stamp_end(p);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -46,6 +50,7 @@ __global__ void __launch_bounds__(128) attn_cc_kernel(const T* __restrict__ q, c
   __shared__ __align__(16) float sK[KT * KS];
   __shared__ __align__(16) float sV[KT * D];
   __shared__ __align__(16) float sQ[16 * D];
+  if (threadIdx.x == 0) stamp_begin(p);
   const int layer = blockIdx.z, h = blockIdx.y, g = h / p.G;
   const int tok0 = blockIdx.x * 16;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -148,14 +153,17 @@ __global__ void __launch_bounds__(128) attn_cc_kernel(const T* __restrict__ q, c
       ob[(static_cast<long long>(tok) * p.Hq + h) * D + lane + 32 * c] = from_f32<T>(acc[r][c] * inv);
     if (lane == 0) lse[static_cast<long long>(tok) * p.Hq + h] = (m[r] + log2f(l[r])) * 0.6931471805599453f;
   }
+  __syncthreads();
+  if (threadIdx.x == 0) stamp_end(p);
 }
 
 // ------------------------------------------------------------------------------------------------
 // a2 score on CUDA cores (Eq. 4): score_j = sum over the w observer rows and the G heads of the
-// group of 2^(s_ij*scale_log2 - lse2_i).  A CTA owns 32 candidate keys; four threads share a key and
-// split the observer rows between them (the sum over rows is the long serial chain otherwise).
-// grid (ceil(n_cand/32), Hkv, nl), block 128, dynamic smem = 32*(D+4)*4 + 32*D*4 + 32*4 bytes.
-static constexpr int kScoreCcKeys = 32;
+// group of 2^(s_ij*scale_log2 - lse2_i).  A CTA owns 8 candidate keys; sixteen threads share a key and
+// split the observer rows between them (the sum over rows is the long serial chain otherwise, and a launch
+// of this path has a few hundred keys at most: many small CTAs, not few long ones).
+// grid (ceil(n_cand/8), Hkv, nl), block 128, dynamic smem = 8*(D+4)*4 + 32*D*4 + 32*4 bytes.
+static constexpr int kScoreCcKeys = 8;
 
 template <typename T, int D>
 __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, const char* __restrict__ cache,
@@ -165,6 +173,7 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
   float* sK = smem_f;                          // [32][KS]
   float* sQ = sK + kScoreCcKeys * KS;          // [32][D]
   float* sL = sQ + 32 * D;                     // [32]
+  if (threadIdx.x == 0) stamp_begin(p);
   const int layer = blockIdx.z, g = blockIdx.y;
   const int key0 = blockIdx.x * kScoreCcKeys;
   const char* blob = cache + layer * p.cache_ls;
@@ -179,7 +188,7 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
     sK[j * KS + c] = key < p.n_cand ? to_f32<T>(Kc[static_cast<long long>(key) * D + c]) : 0.f;
   }
   const int rows = p.w * p.G;
-  const int kj = threadIdx.x >> 2, part = threadIdx.x & 3;       // key of the CTA, quarter of the observer rows
+  const int kj = threadIdx.x >> 4, part = threadIdx.x & 15;     // key of the CTA, sixteenth of the observer rows
   float acc = 0.f;
   const float4* krow = reinterpret_cast<const float4*>(&sK[kj * KS]);
   for (int r0 = 0; r0 < rows; r0 += 32) {
@@ -204,7 +213,7 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
     }
     __syncthreads();
     const int rmax = min(32, rows - r0);
-    for (int r = part; r < rmax; r += 4) {
+    for (int r = part; r < rmax; r += 16) {
       const float4* qrow = reinterpret_cast<const float4*>(&sQ[r * D]);
       float s = 0.f;
 #pragma unroll 8
@@ -217,8 +226,12 @@ __global__ void __launch_bounds__(128) score_cc_kernel(const T* __restrict__ q, 
   }
   acc += __shfl_xor_sync(0xffffffffu, acc, 1);
   acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+  acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+  acc += __shfl_xor_sync(0xffffffffu, acc, 8);
   const int key = key0 + kj;
   if (part == 0 && key < p.n_cand) score[key] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) stamp_end(p);
 }
 
 // ------------------------------------------------------------------------------------------------

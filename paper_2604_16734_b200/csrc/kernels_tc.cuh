@@ -158,6 +158,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       __syncwarp();
       if (lane == 0) {
         pdl_wait();                                // the block's keys were appended by the previous kernel
+        stamp_begin(p);
       }
       if (lane == 0 && Tl > 0) {
         mbar_expect_tx(&sh.q_full[0], NSUB * rows * 128);
@@ -666,6 +667,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     tc_fence_after_sync();
     tmem_dealloc(tmem, TMEM_COLS);
   }
+  if (threadIdx.x == 0) stamp_end(p);
   if (threadIdx.x == 0 && sh.wait_ctl[0]) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
 }
 
@@ -701,6 +703,7 @@ __global__ void __launch_bounds__(128) score_tc_kernel(const __grid_constant__ C
   float* score = reinterpret_cast<float*>(slot + p.score_off) + static_cast<long long>(g) * p.cap;
 
   if (threadIdx.x == 0) {
+    stamp_begin(p);
     mbar_init(&sh.bar_k, 1); mbar_init(&sh.bar_q, 1); mbar_init(&sh.bar_s, 1);
     sh.wait_ctl[0] = 0; sh.wait_ctl[1] = p.wait_limit_k;
     mbar_fence_init();
@@ -781,6 +784,7 @@ __global__ void __launch_bounds__(128) score_tc_kernel(const __grid_constant__ C
     tc_fence_after_sync();
     tmem_dealloc(tmem, TMEM_COLS);
   }
+  if (threadIdx.x == 0) stamp_end(p);
   if (threadIdx.x == 0 && sh.wait_ctl[0]) atomicExch(reinterpret_cast<int*>(ws), -4 /* KVC_ETIMEOUT */);
 }
 

@@ -39,6 +39,10 @@ struct kvc_ctx {
   int wait_limit_k;              // limit of the kernels' waits, in units of 1024 clock cycles
   struct Prof { int kind; cudaEvent_t a, b; };
   std::vector<Prof> prof;
+  // device-side time stamps (kvc_profile_device): the caller's record buffer, its capacity, the kind of every launch so far
+  unsigned long long* stamps_dev;
+  long long stamps_cap;
+  std::vector<int> stamp_kind;
   // KVC_FLAG_ASYNC_COMPRESS: the side streams, per layer an event after its attention and one after its
   // compress kernel, and whether that compress may still be running (host objects, created on first use)
   static constexpr int kSideStreams = 2;     // layers alternate between them: consecutive compress kernels may overlap
@@ -116,6 +120,8 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->encode = nullptr;
   c->use_tc = cfg->dtype == KVC_BF16 && !(cfg->flags & KVC_FLAG_CUDA_CORES);
   c->profiling = false;
+  c->stamps_dev = nullptr;
+  c->stamps_cap = 0;
   c->wait_limit_k = kvc::kDefaultWaitLimitK;
   for (auto& s : c->side) s = nullptr;
   c->pending.assign(cfg->n_layers, 0);
@@ -153,6 +159,47 @@ extern "C" int kvc_profile_read(kvc_ctx* c, double* ms, long long* launches) {
   }
   drop_events(c);
   return rc;
+}
+
+extern "C" int kvc_profile_device(kvc_ctx* c, void* records, long long capacity, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  c->stamp_kind.clear();
+  c->stamps_dev = nullptr;
+  c->stamps_cap = 0;
+  if (!records) return KVC_OK;
+  if (capacity < 1 || (reinterpret_cast<uintptr_t>(records) & 15)) return fail(c, KVC_EINVAL, "records misaligned or capacity < 1");
+  // every record starts as {begin = all ones, end = 0}: the kernels keep the minimum and the maximum
+  cudaError_t e = cudaMemsetAsync(records, 0, (size_t)capacity * 16, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemset2DAsync(records, 16, 0xff, 8, (size_t)capacity, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail(c, KVC_ECUDA, "cudaMemsetAsync(records): %s", cudaGetErrorString(e));
+  c->stamps_dev = (unsigned long long*)records;
+  c->stamps_cap = capacity;
+  return KVC_OK;
+}
+
+extern "C" int kvc_profile_device_read(kvc_ctx* c, const void* records_host, double* ms, long long* launches, double* span_ms) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!records_host || !ms || !launches) return KVC_EINVAL;
+  const unsigned long long* r = (const unsigned long long*)records_host;
+  unsigned long long first = ~0ull, last = 0;
+  for (size_t i = 0; i < c->stamp_kind.size(); ++i) {
+    const unsigned long long b = r[2 * i], e = r[2 * i + 1];
+    if (b == ~0ull || e < b) continue;                    // a launch whose CTAs never stamped (nothing to do)
+    ms[c->stamp_kind[i]] += (double)(e - b) * 1e-6;
+    launches[c->stamp_kind[i]] += 1;
+    if (b < first) first = b;
+    if (e > last) last = e;
+  }
+  if (span_ms) *span_ms = last > first ? (double)(last - first) * 1e-6 : 0.0;
+  c->stamp_kind.clear();
+  return KVC_OK;
+}
+
+// The record of the next launch of the given kind (null when device stamps are off or the buffer is full).
+static unsigned long long* next_stamp(kvc_ctx* c, int kind) {
+  if (!c->stamps_dev || (long long)c->stamp_kind.size() >= c->stamps_cap) return nullptr;
+  c->stamp_kind.push_back(kind);
+  return c->stamps_dev + 2 * (c->stamp_kind.size() - 1);
 }
 
 // Brackets one kernel launch with events when profiling is on.
@@ -615,6 +662,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   // a0 append (the tensor-core attention kernel appends by itself)
   if (!c->use_tc) {
     ProfScope ps(c, 0, st);
+    g.stamps = next_stamp(c, 0);
     dim3 grid((n * g.Hkv + 7) / 8, 1, nl);
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
@@ -629,6 +677,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   // a1 attention
   {
   ProfScope ps(c, 1, st);
+  g.stamps = next_stamp(c, 1);
   if (c->use_tc) {
     int S = 1, R = 2;
     attn_launch_shape(g, !(cf.flags & 4u), &S, &R);
@@ -656,6 +705,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
       // a2 score as a kernel of its own (fp32 on CUDA cores; bf16 with more than 128 observer rows per kv-head:
       // fusing up to 256 rows was measured and is slower, the stand-alone kernel spreads the key tiles wider)
       ProfScope ps(c, 2, st);
+      g.stamps = next_stamp(c, 2);
       if (c->use_tc) {
         e = D == 128 ? launch_tc_score<128>(g, dev, tk, tqo, ws, tok_per_group, st) : launch_tc_score<64>(g, dev, tk, tqo, ws, tok_per_group, st);
       } else if (f32) {
@@ -669,6 +719,7 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     // (a2 +) a3 select + a4 compact
     {
       ProfScope ps(c, 3, st);
+      g.stamps = next_stamp(c, 3);
       if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, st);
       else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, st)
                                          : launch_compress<64, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, st);

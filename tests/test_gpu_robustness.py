@@ -129,3 +129,37 @@ def test_guard_check_notices_a_stray_byte():
     whole[-1] = 1
     with pytest.raises(AssertionError):
         check_guards(kvc, [(whole, view)])
+
+
+# ------------------------------------------------------------------------------------------------
+# device-side time stamps
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_device_time_stamps_count_every_launch(dtype):
+    # every kernel of the stamped calls leaves a record with begin <= end; the records' durations, added per kind,
+    # fit inside the span from the first begin to the last end (the kernels run in stream order), and the results
+    # are those of an unstamped run
+    hq, hkv, d = 8, 2, 128
+    a = Kvc(1, hq, hkv, d, dtype, 256, 160, 16)
+    b = Kvc(1, hq, hkv, d, dtype, 256, 160, 16)
+    torch.manual_seed(11)
+    blocks = [(torch.randn(n, hq, d, device="cuda").to(dtype), torch.randn(n, hkv, d, device="cuda").to(dtype),
+               torch.randn(n, hkv, d, device="cuda").to(dtype)) for n in (160, 150, 160, 33)]
+    before = b.launch_count()
+    b.profile_device(64)
+    p = 0
+    for q, k, v in blocks:
+        oa = a.prefill_chunk(0, q, k, v, p); ob = b.prefill_chunk(0, q, k, v, p)
+        assert torch.equal(oa, ob)
+        p += q.shape[0]
+    ms, cnt, span = b.profile_device_read()
+    b.profile_device(0)
+    assert sum(cnt.values()) == b.launch_count() - before
+    assert cnt["attention"] == 4 and cnt["compress"] == 3
+    assert all(ms[s] > 0 for s in cnt if cnt[s]) and sum(ms.values()) <= span * 1.001
+    assert torch.equal(a.cache_view(0)[2], b.cache_view(0)[2])
+    # off again: the next call must not touch the (freed) record buffer
+    q, k, v = blocks[0]
+    b.prefill_chunk(0, q, k, v, p)
+    torch.cuda.synchronize()
+    assert b.status() == 0

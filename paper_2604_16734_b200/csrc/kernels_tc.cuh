@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     sh.wait_ctl[0] = 0; sh.wait_ctl[1] = p.wait_limit_k;
     mbar_init(&sh.comb_full, 1);
     // key split with one row tile: every other rank of the cluster will copy its partial of this rank's rows here
-    if (S > 1 && !has_B) mbar_expect_tx(&sh.comb_full, (S - 1) * (128 / S) * D * 4);
+    if (S > 1 && !has_B) mbar_expect_tx(&sh.comb_full, (S - 1) * (128 / S) * (D + 4) * 4);
     mbar_fence_init();
   }
   // rows of the Q tiles that TMA never writes (rows >= TOK*G) must still be finite
@@ -277,14 +277,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             mma_commit(&sh.kv_empty[slotK]);
           }
         }
-        if (stored) tma_store_wait_all();            // the appended rows are in the cache before the kernel ends
+        // the stores have read their ring slots (the combine of a key split reuses the ring) ...
+        if (stored) tma_store_wait_read();
       }
     }
     __syncwarp();
+    // Key split with one row tile: softmax group 0 writes over the ring once both key chains are complete, which says
+    // nothing about the stores above; warps 9 and 10 tell it here that no store reads the ring any more.
+    if (S > 1 && !has_B && (warp == 9 || warp == 10)) named_barrier_arrive(6, 128 + 64);
+    if (lane == 0) tma_store_wait_all();        // ... and the appended rows are in the cache before the kernel ends
     if (S > 1) {                                             // the cluster barriers of the combine below
       cluster_arrive(); cluster_wait();
       cluster_arrive(); cluster_wait();
-      if (!has_B) { cluster_arrive(); cluster_wait(); }
     }
   } else {
     reg_inc<216>();
@@ -297,6 +301,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tmem_S = tmem + t * 128 + lane_addr, tmem_O = tmem + 256 + t * 128 + lane_addr;
     float m_ref = -INFINITY, l = 0.f;                        // reference maximum (log2 units) and row sum
+    float wm0 = 1.f, wm1 = 0.f;                              // key split, one row tile: weights of the two key chains' O
     bool ok = true;
     const bool writer = t == 0 || has_B;                     // this group writes results (a row tile of its own)
     const bool active = writer || alt;                       // this group takes part in the key loop
@@ -471,27 +476,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         }
         named_barrier(5, 256);
         if (t == 0 && ok) {
+          // (a key split has one row tile here -- R = 1 -- or two; with one, the rows of chain 1 stay parked and are
+          // folded in when group 0 stages its rows for the cluster: only m and l are merged now)
           const float m1 = sh.stat[2 * r], l1 = sh.stat[2 * r + 1];
-          if (__any_sync(0xffffffffu, m1 != -INFINITY)) {
+          if (m1 != -INFINITY) {
             const float m_all = fmaxf(m_ref, m1);              // group 0 has seen key tile 0, hence a key of every row
-            const float w0 = fast_exp2(m_ref - m_all), w1 = m1 == -INFINITY ? 0.f : fast_exp2(m1 - m_all);
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-              uint32_t o[32];
-              tmem_ld32(tmem_O + c * 32, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const float4 b4 = *reinterpret_cast<const float4*>(mrg + r * D + (((c * 8 + k) ^ (r & 7)) << 2));
-                o[4 * k + 0] = __float_as_uint(fmaf(w1, b4.x, w0 * __uint_as_float(o[4 * k + 0])));
-                o[4 * k + 1] = __float_as_uint(fmaf(w1, b4.y, w0 * __uint_as_float(o[4 * k + 1])));
-                o[4 * k + 2] = __float_as_uint(fmaf(w1, b4.z, w0 * __uint_as_float(o[4 * k + 2])));
-                o[4 * k + 3] = __float_as_uint(fmaf(w1, b4.w, w0 * __uint_as_float(o[4 * k + 3])));
-              }
-              tmem_st32(tmem_O + c * 32, o);
-            }
-            tmem_wait_st();
-            l = fmaf(w1, l1, w0 * l);
+            wm0 = fast_exp2(m_ref - m_all);
+            wm1 = fast_exp2(m1 - m_all);
+            l = fmaf(wm1, l1, wm0 * l);
             m_ref = m_all;
           }
         }
@@ -524,8 +516,120 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         }
       }
     }
-    if (S > 1) {
-      // Combine the partials of the cluster (S is a power of two).  Rank s owns rows [s*rows_per, (s+1)*rows_per)
+    if (S > 1 && !has_B) {
+      // Combine the partials of the cluster, one row tile (S is a power of two; rank s owns rows [s*rows_per,
+      // (s+1)*rows_per)).  Group 0 writes its rows of O -- the two key chains folded together with the weights found
+      // above, chain 1 read from where group 1 parked it -- into a staging tile whose rows carry (m, l) behind the D
+      // values; the rows of every other owner then leave in ONE bulk copy each (shared memory to the owner's shared
+      // memory, completing on a barrier of the owner: this GPU's memory, no multicast), and each rank reduces its rows
+      // from the staging tile (its own partial) and from what the others sent:
+      //   O = sum_s 2^(m_s - m*) O_s / sum_s 2^(m_s - m*) l_s.
+      // Shared memory: the parked rows [128][D] over the Q tiles; over the ring the received rows [S - 1 sources]
+      // [rows_per][D + 4] and the staging tile [128][D + 4] (a row stride of D + 4 floats keeps thread-per-row
+      // accesses off each other's banks).
+      constexpr int RS = D + 4;
+      const int rows_per = 128 / S;
+      const float* mrg = reinterpret_cast<const float*>(smem);
+      float* recv = reinterpret_cast<float*>(smem + 2 * TILE_BYTES);
+      float* stg = recv + (128 - rows_per) * RS;
+      // This CTA's own ring is free: both key chains are complete, the producer loads no tile that is not used, and
+      // the issuer warps arrive on barrier 6 once the stores of the appended tiles have read their slots.
+      if (t == 0) {
+        named_barrier(6, 128 + 64);
+        const bool have = ok && Tl > 0;                         // warp-uniform
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          if (have) {
+            tmem_ld32(tmem_O + c * 32, o);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = 0u;
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            float4 v4 = make_float4(__uint_as_float(o[4 * k]), __uint_as_float(o[4 * k + 1]), __uint_as_float(o[4 * k + 2]), __uint_as_float(o[4 * k + 3]));
+            if (have && alt && wm1 != 0.f) {                  // (0: chain 1 saw no key of the row, or gave up)
+              const float4 b4 = *reinterpret_cast<const float4*>(mrg + r * D + (((c * 8 + k) ^ (r & 7)) << 2));
+              v4.x = fmaf(wm1, b4.x, wm0 * v4.x); v4.y = fmaf(wm1, b4.y, wm0 * v4.y);
+              v4.z = fmaf(wm1, b4.z, wm0 * v4.z); v4.w = fmaf(wm1, b4.w, wm0 * v4.w);
+            }
+            *reinterpret_cast<float4*>(stg + r * RS + (c * 8 + k) * 4) = v4;
+          }
+        }
+        *reinterpret_cast<float4*>(stg + r * RS + D) = make_float4((have && l > 0.f) ? m_ref : -INFINITY, have ? l : 0.f, 0.f, 0.f);
+        fence_proxy_async_smem();                               // the rows just written are read by bulk copies
+      }
+      // Every CTA of the cluster has staged its rows and is done with its ring, where the copies land.  (The barrier
+      // also orders this rank's staged rows before the reads of group 1 below.)
+      cluster_arrive();
+      cluster_wait();
+      if (threadIdx.x == 0) {
+        for (int owner = 0; owner < S; ++owner) {
+          if (owner == split) continue;
+          const int slot = split < owner ? split : split - 1;   // this rank among the owner's other ranks
+          bulk_copy_to_cluster(dsmem_addr(smem_u32(recv + slot * rows_per * RS), owner), smem_u32(stg + owner * rows_per * RS),
+                               rows_per * RS * 4, dsmem_addr(smem_u32(&sh.comb_full), owner));
+        }
+      }
+      ok = mbar_wait(&sh.comb_full, 0, abort_flag) && ok;       // the other ranks' rows have landed
+      {
+        const int r0 = split * rows_per;
+        const int per_tile = rows_per * (D / 32);               // work items: (row, group of 32 columns)
+        for (int item = threadIdx.x; item < per_tile; item += 256) {
+          const int lr = item % rows_per, cg = item / rows_per, r = r0 + lr;
+          const int tok = tokA + r / p.G, hh = r % p.G;
+          if (!(r < rows && tok < p.n)) continue;
+          auto row_of = [&](int s2) -> const float* {
+            return s2 == split ? stg + r * RS : recv + ((s2 < split ? s2 : s2 - 1) * rows_per + lr) * RS;
+          };
+          float m_all = -INFINITY;
+#pragma unroll 1
+          for (int s2 = 0; s2 < S; ++s2) m_all = fmaxf(m_all, row_of(s2)[D]);
+          float L = 0.f;
+          float acc[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll 1
+          for (int s2 = 0; s2 < S; ++s2) {
+            const float* row = row_of(s2);
+            const float2 ml = *reinterpret_cast<const float2*>(row + D);
+            if (ml.x == -INFINITY) continue;                  // this source saw no key of the row
+            const float wt = fast_exp2(ml.x - m_all);
+            L = fmaf(wt, ml.y, L);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const float4 v4 = *reinterpret_cast<const float4*>(row + (cg * 8 + k) * 4);
+              acc[4 * k + 0] = fmaf(wt, v4.x, acc[4 * k + 0]);
+              acc[4 * k + 1] = fmaf(wt, v4.y, acc[4 * k + 1]);
+              acc[4 * k + 2] = fmaf(wt, v4.z, acc[4 * k + 2]);
+              acc[4 * k + 3] = fmaf(wt, v4.w, acc[4 * k + 3]);
+            }
+          }
+          const float inv = 1.f / L;
+          __nv_bfloat16* orow = out + layer * p.out_ls + (static_cast<long long>(tok) * p.Hq + g * p.G + hh) * D + cg * 32;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 vv;
+            vv.x = pack_bf16x2(acc[8 * i + 0] * inv, acc[8 * i + 1] * inv);
+            vv.y = pack_bf16x2(acc[8 * i + 2] * inv, acc[8 * i + 3] * inv);
+            vv.z = pack_bf16x2(acc[8 * i + 4] * inv, acc[8 * i + 5] * inv);
+            vv.w = pack_bf16x2(acc[8 * i + 6] * inv, acc[8 * i + 7] * inv);
+            reinterpret_cast<uint4*>(orow)[i] = vv;
+          }
+          if (cg == 0) {
+            float* lse = reinterpret_cast<float*>(ws_slot(ws, p, layer) + p.lse_off);
+            lse[static_cast<long long>(tok) * p.Hq + g * p.G + hh] = (m_all + log2f(L)) * 0.6931471805599453f;
+          }
+        }
+      }
+      // A CTA must not exit while a bulk copy still reads its staging tile: every rank has waited for the copies
+      // addressed to it, so once all of them are here every copy is complete.
+      cluster_arrive();
+      cluster_wait();
+    } else if (S > 1) {
+      // Combine the partials of the cluster, two row tiles (S is a power of two).  Rank s owns rows [s*rows_per, (s+1)*rows_per)
       // of both tiles.  Tile by tile, the softmax threads park their rows of O (fp32: the output tolerance
       // leaves no room for a 16-bit exchange format) in a local staging tile, then copy it row by row into
       // the owners' shared memory with remote stores -- stores are not waited for, remote loads would be --
@@ -542,10 +646,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
       float* stat = sh.stat;                                    // [S][2][rows_per][2]: m (-inf: row saw no key), l
       cluster_arrive();                                         // every CTA is done with its Q tiles and ring
       cluster_wait();
-      if (writer) {
-        const int nthr = has_B ? 256 : 128;                     // softmax threads that take part
+      {
+        constexpr int nthr = 256;                               // both groups take part
         const bool have = ok && Tl > 0;                         // warp-uniform
-        for (int tt = 0; tt < (has_B ? 2 : 1); ++tt) {
+        for (int tt = 0; tt < 2; ++tt) {
           if (t == tt) {
             const int owner = r / rows_per, lr = r - owner * rows_per;
 #pragma unroll
@@ -566,28 +670,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             if (owner != split) stat_addr = dsmem_addr(stat_addr, owner);
             dsmem_st_v2(stat_addr, (have && l > 0.f) ? m_ref : -INFINITY, have ? l : 0.f);
           }
-          const bool bulk = !has_B;                             // (uniform over the cluster: its CTAs share the row tiles)
-          if (bulk) fence_proxy_async_smem();                   // the rows just written are read by bulk copies
           named_barrier(1, nthr);                               // the staging tile is complete
           constexpr int CPR = D / 4;                            // 16-byte chunks per row
-          if (bulk) {
-            // One row tile: the rows of every other owner leave in ONE bulk copy each (shared memory to the owner's
-            // shared memory, completing on the owner's barrier; this GPU's own memory, no multicast); only this
-            // rank's own rows are copied by the threads.  Per-thread remote stores moved 13 B/clk.
-            if (threadIdx.x == 0) {
-              for (int owner = 0; owner < S; ++owner) {
-                if (owner == split) continue;
-                bulk_copy_to_cluster(dsmem_addr(smem_u32(stage + (split * 2 + tt) * rows_per * D), owner),
-                                     smem_u32(stg + owner * rows_per * D), rows_per * D * 4,
-                                     dsmem_addr(smem_u32(&sh.comb_full), owner));
-              }
-            }
-            for (int idx = threadIdx.x; idx < rows_per * CPR; idx += nthr) {
-              const int lr = idx / CPR, chunk = idx % CPR;
-              *reinterpret_cast<uint4*>(stage + ((split * 2 + tt) * rows_per + lr) * D + chunk * 4) =
-                  *reinterpret_cast<const uint4*>(stg + (split * rows_per + lr) * D + chunk * 4);
-            }
-          } else {
 #pragma unroll 4
           for (int idx = threadIdx.x; idx < 128 * CPR; idx += nthr) {
             const int row = idx / CPR, chunk = idx % CPR;
@@ -597,18 +681,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             if (owner != split) dst = dsmem_addr(dst, owner);
             dsmem_st_v4_b32(dst, v4.x, v4.y, v4.z, v4.w);
           }
-          }
           named_barrier(1, nthr);                               // the staging tile may be overwritten
         }
       }
-      cluster_arrive();                                         // all partials have landed (bulk copies: see below); no
-      cluster_wait();                                           // remote access is started after this
-      // the bulk copies of the other ranks complete on this CTA's barrier, not at the cluster barrier
-      if (!has_B) ok = mbar_wait(&sh.comb_full, 0, abort_flag) && ok;
+      cluster_arrive();                                         // all partials have landed; no remote access is
+      cluster_wait();                                           // started after this
       {
         const int r0 = min(128, split * rows_per), nrows = min(128, r0 + rows_per) - r0;
         const int per_tile = nrows * (D / 32);                  // work items: (row, group of 32 columns)
-        for (int item = threadIdx.x; item < (has_B ? 2 : 1) * per_tile; item += 256) {
+        for (int item = threadIdx.x; item < 2 * per_tile; item += 256) {
           const int t = item / per_tile, rem = item % per_tile;
           const int lr = rem % nrows, cg = rem / nrows, r = r0 + lr;
           const int tok = (t ? tokB : tokA) + r / p.G, hh = r % p.G;
@@ -655,9 +736,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           }
         }
       }
-      // A CTA must not exit while a bulk copy still reads its staging tile: every rank has waited for the copies
-      // addressed to it, so once all of them are here every copy is complete.
-      if (!has_B) { cluster_arrive(); cluster_wait(); }
     }
   }
 

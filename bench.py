@@ -364,6 +364,7 @@ class Runner:
         for p, n in self.sched:
             for l in range(self.L):
                 kv.prefill_chunk_host(l, qh[l, p:p + n], kh[l, p:p + n], vh[l, p:p + n], p, oh[l, p:p + n])
+        kv.host_flush()                                       # the step ends when the last result is on the host
 
 
 def max_over_ranks(seconds: float, dist, device) -> float:

@@ -166,14 +166,22 @@ int kvc_staging_nbytes(const kvc_ctx* ctx, size_t* nbytes);
 
 /* kvc_prefill_chunk with HOST q/k/v/out (pinned memory recommended): copies the block's q, k, v
  * into `staging` (DEVICE, kvc_staging_nbytes bytes, 256-byte aligned), runs the block, copies `out`
- * back to the host.  Nothing blocks the host; out_host is valid, and the host inputs may be reused, after
- * `stream` is synchronised.  Consecutive calls alternate between the two halves of `staging`: the
- * host-to-device copies of a call run on a stream the context owns and `stream` waits for them, so they
- * overlap the previous call's kernels and device-to-host copy (pass the same `staging` to every call of a
- * context; a run-time error before the kernels leaves the call without effect on the cache). */
+ * back to the host.  Nothing blocks the host.  Consecutive calls alternate between the two halves of
+ * `staging`; the copies in either direction run on two streams the context owns: the host-to-device copies of a
+ * call start as soon as the block that last used its half is done and `stream` waits for them before the kernels,
+ * the device-to-host copy of `out` follows the kernels, and `stream` waits for it only behind the NEXT call's
+ * kernels.  So the inbound copies, the kernels and the outbound copy of three consecutive calls overlap.
+ * The host inputs of a call may be reused once `stream` has completed the call.  out_host of a call is complete
+ * once `stream` has completed the next kvc_prefill_chunk_host call of the context, or a kvc_host_flush after the
+ * call.  (Pass the same `staging` to every call of a context; a run-time error before the kernels leaves the call
+ * without effect on the cache.) */
 int kvc_prefill_chunk_host(kvc_ctx* ctx, int layer, const void* q_host, const void* k_host,
                            const void* v_host, int n, long long pos0, void* cache, void* workspace,
                            void* staging, void* out_host, void* stream);
+
+/* Makes `stream` wait for the device-to-host copies of all kvc_prefill_chunk_host calls made so far (no host wait;
+ * nothing is enqueued when there was none): once `stream` has completed, every out_host is filled. */
+int kvc_host_flush(kvc_ctx* ctx, void* stream);
 
 /* (No counterpart in the paper: an integration convenience.)
  * kvc_prefill_chunk for callers that have no way to obtain scratch memory: code running where

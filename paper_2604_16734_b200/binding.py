@@ -22,7 +22,7 @@ KVC_FLAG_ASYNC_COMPRESS = 16
 
 EXPORTS = [
     "kvc_create", "kvc_destroy", "kvc_cache_nbytes", "kvc_workspace_init", "kvc_reset",
-    "kvc_prefill_chunk", "kvc_prefill_chunk_layers", "kvc_staging_nbytes", "kvc_prefill_chunk_host",
+    "kvc_prefill_chunk", "kvc_prefill_chunk_layers", "kvc_staging_nbytes", "kvc_prefill_chunk_host", "kvc_host_flush",
     "kvc_prefill_chunk_static", "kvc_status_static", "kvc_prefill_chunk_proxy",
     "kvc_join", "kvc_cache_view", "kvc_workspace_view", "kvc_move_counts", "kvc_status", "kvc_kv_bytes", "kvc_profile_enable",
     "kvc_profile_read", "kvc_launch_count", "kvc_last_error", "kvc_set_wait_limit", "kvc_selftest_wait_timeout",
@@ -63,6 +63,7 @@ def load_library() -> ctypes.CDLL:
     lib.kvc_prefill_chunk_layers.argtypes = [vp, i, i, vp, ll, vp, vp, ll, i, ll, vp, sz, vp, vp, ll, vp]
     lib.kvc_staging_nbytes.argtypes = [vp, psz]
     lib.kvc_prefill_chunk_host.argtypes = [vp, i, vp, vp, vp, i, ll, vp, vp, vp, vp, vp]
+    lib.kvc_host_flush.argtypes = [vp, vp]
     lib.kvc_prefill_chunk_static.argtypes = [vp, i, vp, vp, vp, i, ll, vp, vp, vp]
     lib.kvc_status_static.argtypes = [vp, vp]
     lib.kvc_cache_view.argtypes = [vp, i, vp, ctypes.POINTER(KvcView)]
@@ -206,7 +207,8 @@ class Kvc:
 
     def prefill_chunk_host(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, pos0: int,
                            out: torch.Tensor) -> torch.Tensor:
-        """q/k/v/out are HOST tensors (pinned for asynchronous copies)."""
+        """q/k/v/out are HOST tensors (pinned for asynchronous copies).  ``out`` is complete once the stream has run
+        the next call of this method or ``host_flush``."""
         if self.staging is None:
             self.staging = torch.empty(self.staging_bytes, dtype=torch.uint8, device=self.device)
         assert not q.is_cuda and not out.is_cuda
@@ -214,6 +216,10 @@ class Kvc:
                                                      self.cache[layer].data_ptr(), self.workspace.data_ptr(),
                                                      self.staging.data_ptr(), _ptr(out), self._stream()))
         return out
+
+    def host_flush(self) -> None:
+        """The current stream waits for the copies of every ``out`` of ``prefill_chunk_host`` so far."""
+        self._check(self._lib.kvc_host_flush(self._h, self._stream()))
 
     def prefill_chunk_static(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, pos0: int,
                              out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -35,6 +35,7 @@ static constexpr int kRankMax = 256;          // keys of the cut-off bin that ar
 static constexpr int kMaxKeysSmem = 6144;     // candidates whose keys fit the shared-memory table (48 KB)
 static constexpr int kMaxMovesSmem = 2048;    // moves whose (src, dst) fit the shared-memory tables (16 KB)
 static constexpr int kMaxObsRowsFused = 128;  // observer rows (w * G) the fused scoring phase takes
+static constexpr int kMaxClusterWide = 16;   // largest cluster the host asks for (non-portable size: more than 8 CTAs)
 static constexpr int kScoresGiven = 0, kScoreAttention = 1, kScoreKeyDiff = 2;   // what phase 1 of compress_kernel does
 static constexpr int kSubTileBytesC = 128 * 128;
 

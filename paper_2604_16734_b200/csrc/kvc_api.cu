@@ -51,8 +51,8 @@ struct kvc_ctx {
   std::vector<char> pending;
   // kvc_prefill_chunk_host: the stream that carries the host-to-device copies, per staging half an event after its
   // copies (recorded there) and one after the block that read it (recorded on the caller's stream); call counter
-  cudaStream_t copy_in;
-  cudaEvent_t ev_in[2], ev_free[2];
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t ev_in[2], ev_free[2], ev_out[2];
   unsigned host_calls;
   char err[512];
 };
@@ -125,8 +125,8 @@ extern "C" int kvc_create(const kvc_config* cfg, kvc_ctx** out) {
   c->wait_limit_k = kvc::kDefaultWaitLimitK;
   for (auto& s : c->side) s = nullptr;
   c->pending.assign(cfg->n_layers, 0);
-  c->copy_in = nullptr;
-  for (int i = 0; i < 2; ++i) { c->ev_in[i] = nullptr; c->ev_free[i] = nullptr; }
+  c->copy_in = c->copy_out = nullptr;
+  for (int i = 0; i < 2; ++i) { c->ev_in[i] = nullptr; c->ev_free[i] = nullptr; c->ev_out[i] = nullptr; }
   c->host_calls = 0;
   c->err[0] = 0;
   *out = c;
@@ -258,11 +258,13 @@ extern "C" int kvc_destroy(kvc_ctx* c) {
     for (auto ev : c->ev_comp) if (ev) cudaEventDestroy(ev);
     c->ev_attn.clear(); c->ev_comp.clear();
     for (auto& s : c->side) { if (s) cudaStreamDestroy(s); s = nullptr; }
+    if (c->copy_out) { cudaStreamSynchronize(c->copy_out); cudaStreamDestroy(c->copy_out); c->copy_out = nullptr; }
     if (c->copy_in) { cudaStreamSynchronize(c->copy_in); cudaStreamDestroy(c->copy_in); c->copy_in = nullptr; }
     for (int i = 0; i < 2; ++i) {
       if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
       if (c->ev_free[i]) cudaEventDestroy(c->ev_free[i]);
-      c->ev_in[i] = c->ev_free[i] = nullptr;
+      if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
+      c->ev_in[i] = c->ev_free[i] = c->ev_out[i] = nullptr;
     }
   }
   drop_events(c);
@@ -517,17 +519,45 @@ static cudaError_t launch_tc_attn(const Geom& g, int dev, const CUtensorMap& tq,
 // a2..a4 fused (compress.cuh).  MODE: kvc::kScoresGiven / kScoreAttention / kScoreKeyDiff.
 template <int D, int MODE>
 static cudaError_t launch_compress(const Geom& g, int dev, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
-                                   int elem_bytes, bool pdl, cudaStream_t st) {
+                                   int elem_bytes, bool pdl, bool wide_ok, cudaStream_t st) {
   const int score_bytes = MODE == kvc::kScoreAttention ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * kvc::kMaxObsRowsFused * 128 : 0;
   const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4 + 2 * kvc::kSelBins * 4;   // keys, move tables, histograms
   const int smem_min = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
   const int smem_solo = 120 * 1024;                      // more than half an SM: one CTA per SM
   static bool attr_set[kMaxDevices] = {};
   if (cudaError_t e = opt_in_smem(kvc::compress_kernel<D, MODE>, smem_solo, attr_set, dev)) return e;
+  // Clusters of more than 8 CTAs are not portable: the kernel must allow them, and the device says how many clusters
+  // of a size (one CTA per SM) it can hold at a time -- asked once per device and size; 0 where it refuses.
+  static int wide_clusters[kMaxDevices][kvc::kMaxClusterWide + 1] = {};   // 0: not asked yet, -1: none, else clusters in flight
+  auto clusters_in_flight = [&](int size) {
+    int& slot = wide_clusters[dev][size];
+    if (slot == 0) {
+      int n_wide = 0;
+      if (cudaFuncSetAttribute(kvc::compress_kernel<D, MODE>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+        cudaLaunchConfig_t q;
+        memset(&q, 0, sizeof(q));
+        q.gridDim = dim3(size, 1, 1);
+        q.blockDim = dim3(kvc::kCompressThreads, 1, 1);
+        q.dynamicSmemBytes = smem_solo;
+        LaunchAttrs qa(size, false);
+        q.attrs = qa.at;
+        q.numAttrs = qa.n;
+        if (cudaOccupancyMaxActiveClusters(&n_wide, kvc::compress_kernel<D, MODE>, &q) != cudaSuccess) n_wide = 0;
+      }
+      (void)cudaGetLastError();                           // a refusal is an answer, not an error of this call
+      slot = n_wide > 0 ? n_wide : -1;
+    }
+    return slot;
+  };
   // cluster size: spread one kv-head over several SMs when the heads alone cannot fill the GPU
   const int n_tiles = (g.n_cand + 127) / 128;
   int Cn = (int)(kvc::kNumSMs / ((long long)g.Hkv * g.nl));
-  if (Cn > 8) Cn = 8;                                     // portable cluster size limit
+  if (Cn > kvc::kMaxClusterWide) Cn = kvc::kMaxClusterWide;
+  // More than the portable 8 CTAs only while every cluster of the launch can be resident at once, and only in stream
+  // order: on a side stream the kernel shares the GPU with the next layer's attention, where a wider cluster waits
+  // longer for its SMs than it saves (measured: the video workload's step went from 44 to 49 ms).
+  if (!wide_ok && Cn > 8) Cn = 8;
+  while (Cn > 8 && clusters_in_flight(Cn) < (long long)g.Hkv * g.nl) --Cn;
   const int tiles_per_cta = 2;                            // fewer, and the cluster barriers cost more than the tiles
   if (Cn > (n_tiles + tiles_per_cta - 1) / tiles_per_cta) Cn = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
   if (Cn < 1) Cn = 1;
@@ -720,10 +750,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     {
       ProfScope ps(c, 3, st);
       g.stamps = next_stamp(c, 3);
-      if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, st);
-      else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, st)
-                                         : launch_compress<64, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, st);
-      else e = launch_compress<64, kvc::kScoresGiven>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, st);
+      if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, !async_compress, st);
+      else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, !async_compress, st)
+                                         : launch_compress<64, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, !async_compress, st);
+      else e = launch_compress<64, kvc::kScoresGiven>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, !async_compress, st);
     }
     if (e != cudaSuccess) return check_cuda(c, e, "compress launch");
     c->launches++;
@@ -780,8 +810,13 @@ static int ensure_copy_stream(kvc_ctx* c) {
   for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
     if (!c->ev_in[i] && (e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming)) != cudaSuccess) c->ev_in[i] = nullptr;
     if (e == cudaSuccess && !c->ev_free[i] && (e = cudaEventCreateWithFlags(&c->ev_free[i], cudaEventDisableTiming)) != cudaSuccess) c->ev_free[i] = nullptr;
+    if (e == cudaSuccess && !c->ev_out[i] && (e = cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming)) != cudaSuccess) c->ev_out[i] = nullptr;
   }
   if (e != cudaSuccess) return fail(c, KVC_ECUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+  if (!c->copy_out && (e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking)) != cudaSuccess) {
+    c->copy_out = nullptr;
+    return fail(c, KVC_ECUDA, "cudaStreamCreate: %s", cudaGetErrorString(e));
+  }
   if ((e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking)) != cudaSuccess) {
     c->copy_in = nullptr;
     return fail(c, KVC_ECUDA, "cudaStreamCreate: %s", cudaGetErrorString(e));
@@ -805,9 +840,12 @@ extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host,
   kvc_staging_nbytes(c, &total);
   int rc = ensure_copy_stream(c);
   if (rc) return rc;
-  // Calls alternate between the two halves of the staging buffer.  The inputs travel on the context's copy stream,
-  // behind the block that last read this half (two calls ago), so they overlap the previous call's kernels and its
-  // device-to-host copy; the caller's stream waits for them, runs the block and copies `out` back.
+  // Calls alternate between the two halves of the staging buffer.  The inputs travel on the context's inbound copy
+  // stream, behind the block that last read this half (two calls ago); the caller's stream waits for them and runs
+  // the block; `out` goes back on the context's outbound copy stream, behind the block.  So the inbound copies of
+  // call i+1, the kernels of call i+1 (other half) and the outbound copy of call i all run at the same time.  The
+  // caller's stream then waits for the outbound copy of the PREVIOUS call (the other half: its `out` area is the
+  // next block's), which has had this call's kernels to finish.
   const int half = (int)(c->host_calls++ & 1u);
   char* dq = (char*)staging + half * (total / 2);
   char* dk = dq + align_up(qb, 256);
@@ -822,7 +860,19 @@ extern "C" int kvc_prefill_chunk_host(kvc_ctx* c, int layer, const void* q_host,
   rc = run_chunk(c, layer, 1, dq, 0, dk, dv, 0, n, pos0, cache, 0, workspace, dout, 0, st, 0, false);   // staging is reused: no side stream
   if (rc) return rc;
   if ((rc = check_cuda(c, cudaEventRecord(c->ev_free[half], st), "cudaEventRecord"))) return rc;
-  return check_cuda(c, cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st), "D2H out");
+  if ((rc = check_cuda(c, cudaStreamWaitEvent(c->copy_out, c->ev_free[half], 0), "cudaStreamWaitEvent"))) return rc;
+  if ((rc = check_cuda(c, cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, c->copy_out), "D2H out"))) return rc;
+  if ((rc = check_cuda(c, cudaEventRecord(c->ev_out[half], c->copy_out), "cudaEventRecord"))) return rc;
+  // (an event that was never recorded counts as complete: the first call waits for nothing here)
+  return check_cuda(c, cudaStreamWaitEvent(st, c->ev_out[1 - half], 0), "cudaStreamWaitEvent");
+}
+
+extern "C" int kvc_host_flush(kvc_ctx* c, void* stream) {
+  if (!live(c)) return KVC_ESTATE;
+  if (!c->copy_out) return KVC_OK;                           // no host call yet
+  for (int i = 0; i < 2; ++i)
+    if (int rc = check_cuda(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_out[i], 0), "cudaStreamWaitEvent")) return rc;
+  return KVC_OK;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -501,9 +501,40 @@ def test_host_buffer_entry_point():
     for pos0, n in cfg.chunks():
         ref = a.prefill_chunk(0, q[pos0:pos0 + n].cuda(), k[pos0:pos0 + n].cuda(), v[pos0:pos0 + n].cuda(), pos0)
         b.prefill_chunk_host(0, qh[pos0:pos0 + n], kh[pos0:pos0 + n], vh[pos0:pos0 + n], pos0, out_h[pos0:pos0 + n])
-        torch.cuda.synchronize()
+        b.host_flush()
+        torch.cuda.current_stream().synchronize()
         assert torch.equal(ref.cpu(), out_h[pos0:pos0 + n])
     assert torch.equal(a.cache_view(0)[2], b.cache_view(0)[2])
+
+
+def test_host_buffer_entry_point_back_to_back():
+    # Calls enqueued without waiting in between: the copies of three consecutive calls overlap, the staging halves
+    # alternate, and one flush at the end must be enough for every result (several layers, two passes over the same
+    # host buffers with the results cleared in between).
+    cfg = reduced(CONFIGS["C4"], n_layers=3, n_units=14)          # 2744 vision tokens > B = 2048: the last blocks evict
+    wl = Workload(cfg)
+    layers = [wl.layer(l) for l in range(3)]
+    a = _kvc_for(cfg); b = _kvc_for(cfg)
+    refs = [torch.empty_like(layers[l][0]) for l in range(3)]
+    for pos0, n in cfg.chunks():
+        for l, (q, k, v) in enumerate(layers):
+            refs[l][pos0:pos0 + n] = a.prefill_chunk(l, q[pos0:pos0 + n].cuda(), k[pos0:pos0 + n].cuda(), v[pos0:pos0 + n].cuda(), pos0).cpu()
+    pinned = [tuple(t.pin_memory() for t in layers[l]) for l in range(3)]
+    outs = [torch.empty_like(layers[l][0]).pin_memory() for l in range(3)]
+    for _ in range(2):
+        b.reset()
+        for o in outs:
+            o.zero_()
+        for pos0, n in cfg.chunks():
+            for l, (qh, kh, vh) in enumerate(pinned):
+                b.prefill_chunk_host(l, qh[pos0:pos0 + n], kh[pos0:pos0 + n], vh[pos0:pos0 + n], pos0, outs[l][pos0:pos0 + n])
+        b.host_flush()
+        torch.cuda.current_stream().synchronize()
+        assert b.status() == 0
+        for l in range(3):
+            assert torch.equal(refs[l], outs[l])
+    for l in range(3):
+        assert torch.equal(a.cache_view(l)[2], b.cache_view(l)[2])
 
 
 def test_argument_errors_enqueue_nothing():

@@ -260,19 +260,43 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           tc_fence_after_sync();
           issue_PV(slotV, 0, it > 0);
           const bool hold_v = append_item(iv, slotV);
+          // What follows the second half of P is the row tile's critical chain (P -> P V -> next S -> softmax).  With
+          // two row tiles nothing else sits between the two groups of MMAs: the next K tile (landed long ago) is
+          // waited for here, and the commits that free the slots and publish O come after the next S has been issued
+          // (they then complete with it, which nobody minds: O is read after the next S at the earliest).  In-kernel
+          // stamps put the commits and the wait at 380 of the chain's 4000 cycles.  With one row tile and two key
+          // chains every ring item feeds one chain only and the ring holds one key tile per chain: there the V slot
+          // goes back to the producer first, and the K tile is waited for when it is needed (measured: the deferred
+          // order starves the other chain and costs 13 %).
+          const bool defer = !alt;
+          if (defer && jn < Tl) {
+            ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
+            if (!ok) break;
+          }
           ok = mbar_wait(&sh.p_half[t][1], it & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           issue_PV(slotV, 1, true);
-          mma_commit(&sh.pv_done[t]);
-          if (hold_v) tma_store_wait_read();
-          mma_commit(&sh.kv_empty[slotV]);
+          if (!defer) {
+            mma_commit(&sh.pv_done[t]);
+            if (hold_v) tma_store_wait_read();
+            mma_commit(&sh.kv_empty[slotV]);
+            if (jn < Tl) {
+              ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after_sync();
+            }
+          }
           if (jn < Tl) {
-            ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after_sync();
             issue_S(slotK);
             mma_commit(&sh.s_full[t]);
+          }
+          if (defer) {
+            mma_commit(&sh.pv_done[t]);
+            if (hold_v) tma_store_wait_read();
+            mma_commit(&sh.kv_empty[slotV]);
+          }
+          if (jn < Tl) {
             if (append_item(ik, slotK)) tma_store_wait_read();
             mma_commit(&sh.kv_empty[slotK]);
           }

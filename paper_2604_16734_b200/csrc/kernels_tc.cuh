@@ -355,16 +355,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           for (int c = 0; c < 128; ++c)
             if (c >= lim) sr[c] = 0xff800000u;                // -inf
         }
-        float mx4[8];                                         // independent chains: latency, not issue, is the cost
+        float mx4[8];                                         // independent chains of three-input maxima
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mx4[i] = __uint_as_float(sr[i]);
+        for (int i = 0; i < 8; ++i) mx4[i] = fmaxf(__uint_as_float(sr[i]), __uint_as_float(sr[8 + i]));
 #pragma unroll
-        for (int c = 8; c < 128; c += 8) {
+        for (int c = 16; c < 128; c += 16) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sr[c + i]));
+          for (int i = 0; i < 8; ++i) mx4[i] = fmax3(mx4[i], __uint_as_float(sr[c + i]), __uint_as_float(sr[c + 8 + i]));
         }
-        const float mx = fmaxf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])),
-                               fmaxf(fmaxf(mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
+        const float mx = fmaxf(fmax3(mx4[0], mx4[1], mx4[2]), fmaxf(fmax3(mx4[3], mx4[4], mx4[5]), fmaxf(mx4[6], mx4[7])));
         const float m_new = mx * p.scale_log2;                // scale > 0
         if (it == 0) {
           m_ref = m_new == -INFINITY ? 0.f : m_new;
@@ -390,17 +389,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
         // Only the exponentials are taken in turns: loading S and finding the row maxima overlap the other
         // tile's exponentials.
         if (turns) { named_barrier(2 + t, 256); took_turn = true; }
-        const float neg_m = -m_ref;
-        float ps[4] = {0.f, 0.f, 0.f, 0.f};
+        // (packed fp32: one instruction scales two columns, one adds two exponentials to the partial sums)
+        const uint64_t scale2 = f32x2(p.scale_log2, p.scale_log2), neg_m2 = f32x2(-m_ref, -m_ref);
+        uint64_t ps2[2] = {f32x2(0.f, 0.f), f32x2(0.f, 0.f)};
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i]), p.scale_log2, neg_m));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sr[c * 32 + 2 * i + 1]), p.scale_log2, neg_m));
-            ps[(i & 1) * 2] += p0;
-            ps[(i & 1) * 2 + 1] += p1;
+            float x0, x1;
+            f32x2_split(fma_f32x2(f32x2(__uint_as_float(sr[c * 32 + 2 * i]), __uint_as_float(sr[c * 32 + 2 * i + 1])), scale2, neg_m2), x0, x1);
+            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+            ps2[i & 1] = add_f32x2(ps2[i & 1], f32x2(p0, p1));
             pk[i] = pack_bf16x2(p0, p1);
           }
           tmem_st16(tmem_S + c * 16, pk);
@@ -410,7 +410,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             mbar_arrive(&sh.p_half[t][c >> 1]);
           }
         }
-        l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
+        {
+          float ps[4];
+          f32x2_split(ps2[0], ps[0], ps[1]);
+          f32x2_split(ps2[1], ps[2], ps[3]);
+          l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
+        }
         } while (0);
         if (turns && !took_turn) named_barrier(2 + t, 256);   // a wait gave up before the turn was taken: take it now
         // hand the turn over if the other group has a key tile left: its it-th (group 0 asks) or (it+1)-th (group 1)

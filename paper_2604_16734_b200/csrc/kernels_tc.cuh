@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.q_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.pv_done[i], 1);
-      mbar_init(&sh.p_half[i][0], 128); mbar_init(&sh.p_half[i][1], 128);
+      mbar_init(&sh.p_half[i][0], 4); mbar_init(&sh.p_half[i][1], 4);     // one arrival per softmax warp
     }
     // a ring slot is free again once the issuer of every active row tile has committed its MMAs on it
     for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], has_B ? 2 : 1); }
@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           const int jn = jj + step;                  // the key tile whose S is queued behind P V of this one
           const int iv = 2 * jj + 1, ik = 2 * jn;
           const int slotV = iv % kStages, slotK = ik % kStages;
-          ok = mbar_wait(&sh.p_half[t][0], it & 1, abort_flag) && mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
+          ok = mbar_wait_spin(&sh.p_half[t][0], it & 1, abort_flag) && mbar_wait(&sh.kv_full[slotV], (iv / kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           issue_PV(slotV, 0, it > 0);
@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
             ok = mbar_wait(&sh.kv_full[slotK], (ik / kStages) & 1, abort_flag);
             if (!ok) break;
           }
-          ok = mbar_wait(&sh.p_half[t][1], it & 1, abort_flag);
+          ok = mbar_wait_spin(&sh.p_half[t][1], it & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           issue_PV(slotV, 1, true);
@@ -407,7 +407,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_tc_kernel(const __grid_c
           if (c & 1) {                                        // 64 keys of P are in TMEM: release them to the MMA warp
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(&sh.p_half[t][c >> 1]);
+            // one arrival per warp: 128 arrivals on one shared-memory word are served one after the other, and the
+            // issuer saw the barrier complete some 300 cycles after the first of them (in-kernel stamps)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.p_half[t][c >> 1]);
           }
         }
         {

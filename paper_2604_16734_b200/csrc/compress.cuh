@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
     const int n_mma = (cols + 15) & ~15;
     if (tid == 0) {
       mbar_init(&sh.q_full, 1);
-      for (int i = 0; i < 2; ++i) { mbar_init(&sh.k_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.t_free[i], 128); }
+      for (int i = 0; i < 2; ++i) { mbar_init(&sh.k_full[i], 1); mbar_init(&sh.s_full[i], 1); mbar_init(&sh.t_free[i], 4); }
       mbar_fence_init();
     }
     // observer rows beyond the real ones are padding: keep them finite
@@ -190,7 +190,8 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
         }
         acc += acc2;
         tc_fence_before_sync();
-        mbar_arrive(&sh.t_free[b]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.t_free[b]);              // one arrival per warp of the epilogue group
         const int key = (rank + i * Cn) * 128 + (warp & 3) * 32 + lane;
         if (key < p.n_cand) score[key] = acc;
       }

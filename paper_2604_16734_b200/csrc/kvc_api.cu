@@ -471,7 +471,7 @@ struct LaunchAttrs {
 // Launch shape of the tensor-core attention: R row tiles per CTA (1 or 2) and the key split S over a cluster.
 // For each R the split is the largest that the SM count, the portable cluster size and the rule of three key
 // tiles per CTA allow; the two candidates are then compared with a model of the kernel's duration fitted to
-// in-kernel time stamps (us): a key tile costs 2.1 per pair of row tiles taking turns and 1.15 for a single
+// in-kernel time stamps (us): a key tile costs 1.8 per pair of row tiles taking turns and 1.15 for a single
 // tile (whose two softmax groups take alternate key tiles); the combine costs 3.5 for its barriers and the reduce plus 3.6 per row tile for the remote stores of a
 // whole tile's partial rows; CTAs beyond one per SM run as further waves.
 static void attn_launch_shape(const Geom& g, bool allow_split, int* S_out, int* R_out) {
@@ -488,7 +488,7 @@ static void attn_launch_shape(const Geom& g, bool allow_split, int* S_out, int* 
     if (S < 1) S = 1;
     const int Tl = (T + S - 1) / S;
     const long long waves = (base * S + kvc::kNumSMs - 1) / kvc::kNumSMs;
-    double est = Tl * (R == 2 ? 2.1 : 1.15) * (double)waves;
+    double est = Tl * (R == 2 ? 1.8 : 1.15) * (double)waves;
     if (S > 1) est += 3.5 + R * 3.6 * (S - 1) / S;
     if (R == 2 || est < best) { best = est; *S_out = S; *R_out = R; }
     if (tiles == 1) break;               // a single row tile: both shapes are the same launch

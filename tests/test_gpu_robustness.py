@@ -82,6 +82,36 @@ def test_query_agnostic_score_identical_keys_keep_the_oldest(dtype, d):
 
 
 # ------------------------------------------------------------------------------------------------
+# scores that leave the running maximum far behind
+
+@pytest.mark.parametrize("hq,hkv,blocks", [(2, 2, (512, 512)), (8, 2, (256, 200, 256)), (4, 1, (128, 128, 128, 77))])
+def test_a_key_whose_score_dwarfs_everything_before_it(hq, hkv, blocks):
+    # The attention kernel keeps a reference maximum per row and raises it (rescaling O and the row sum) only when a
+    # tile's maximum exceeds it by more than a threshold.  Here every query is the same +-1 vector u, ordinary keys
+    # are small, and a few keys are large multiples of u, each larger than the last, placed in the first and in the
+    # second half of key tiles that are not a row's first: their scores (5 |u|^2 / sqrt(d) = 57 nats and up) exceed
+    # everything before them by far more than any lazy rule may let pass, for the rows that can see them and not for
+    # the others of the same warp.  The softmax saturates on those keys; outputs, scores and retained sets must match.
+    d, B, w = 128, 1024, 8
+    kvc = Kvc(1, hq, hkv, d, torch.bfloat16, B, max(blocks), w)
+    orc = KVCOracle(1, hq, hkv, d, B, w)
+    g = torch.Generator().manual_seed(7)
+    u = (torch.randint(0, 2, (d,), generator=g) * 2 - 1).float()
+    big = {200: 5.0, 300: 8.0, 470: 12.0, 600: 16.0, 900: 24.0}     # token -> multiple of u (tile halves: 2nd, 1st, 2nd, 2nd, 1st)
+    p = 0
+    for n in blocks:
+        q = u.expand(n, hq, d).clone().bfloat16()
+        k = (0.25 * torch.randn(n, hkv, d, generator=g)).bfloat16()
+        v = torch.randn(n, hkv, d, generator=g).bfloat16()
+        for tok, mult in big.items():
+            if p <= tok < p + n:
+                k[tok - p] = (mult * u).bfloat16()
+        stats = compare_chunk(kvc, orc, 0, q, k, v, p)
+        assert kvc.status() == 0
+        p += n
+    assert stats is not None
+
+# ------------------------------------------------------------------------------------------------
 # the bounded wait
 
 def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():

@@ -519,7 +519,7 @@ static cudaError_t launch_tc_attn(const Geom& g, int dev, const CUtensorMap& tq,
 // a2..a4 fused (compress.cuh).  MODE: kvc::kScoresGiven / kScoreAttention / kScoreKeyDiff.
 template <int D, int MODE>
 static cudaError_t launch_compress(const Geom& g, int dev, const CUtensorMap& tk, const CUtensorMap& tqo, void* cache, void* ws,
-                                   int elem_bytes, bool pdl, bool wide_ok, cudaStream_t st) {
+                                   int elem_bytes, bool pdl, bool wide_ok, int cn_cap, cudaStream_t st) {
   const int score_bytes = MODE == kvc::kScoreAttention ? 2 * (D / 64) * kvc::kSubTileBytesC + (D / 64) * kvc::kMaxObsRowsFused * 128 : 0;
   const int table_bytes = kvc::kMaxKeysSmem * 8 + 2 * kvc::kMaxMovesSmem * 4 + 2 * kvc::kSelBins * 4;   // keys, move tables, histograms
   const int smem_min = (score_bytes > table_bytes ? score_bytes : table_bytes) + 1024;
@@ -557,6 +557,7 @@ static cudaError_t launch_compress(const Geom& g, int dev, const CUtensorMap& tk
   // order: on a side stream the kernel shares the GPU with the next layer's attention, where a wider cluster waits
   // longer for its SMs than it saves (measured: the video workload's step went from 44 to 49 ms).
   if (!wide_ok && Cn > 8) Cn = 8;
+  if (cn_cap > 0 && Cn > cn_cap) Cn = cn_cap;             // (side stream: stay within the SMs the attention leaves idle)
   while (Cn > 8 && clusters_in_flight(Cn) < (long long)g.Hkv * g.nl) --Cn;
   const int tiles_per_cta = 2;                            // fewer, and the cluster barriers cost more than the tiles
   if (Cn > (n_tiles + tiles_per_cta - 1) / tiles_per_cta) Cn = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
@@ -705,12 +706,15 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
   }
   if (e != cudaSuccess) return check_cuda(c, e, "append launch");
   // a1 attention
+  long long attn_ctas = 0;                                    // CTAs of the attention launch (tensor-core path)
   {
   ProfScope ps(c, 1, st);
   g.stamps = next_stamp(c, 1);
   if (c->use_tc) {
     int S = 1, R = 2;
     attn_launch_shape(g, !(cf.flags & 4u), &S, &R);
+    const int TOK = 128 / g.G;
+    attn_ctas = (long long)(((g.n + TOK - 1) / TOK + R - 1) / R) * S * g.Hkv * g.nl;
     e = D == 128 ? launch_tc_attn<128>(g, dev, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st)
                  : launch_tc_attn<64>(g, dev, tq, tk, tv, tkin, tvin, cache, out, ws, S, R, pdl, st);
   } else if (f32) {
@@ -729,6 +733,13 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
       st = c->side[layer0 % kvc_ctx::kSideStreams];                                           // everything below goes to the side stream
     }
     const bool pdl = pdl_main && !async_compress;             // an event, not a kernel, precedes the side stream's launches
+    // On a side stream the kernel runs beside the next layer's attention, a launch of the same shape as this
+    // layer's: a cluster per kv-head that fits the SMs that launch leaves idle shares nothing with it, while a wider
+    // one takes SMs from attention CTAs, which then start late and lengthen the launch everything else waits for
+    // (measured on the video workload: 44.3 -> 39.5 ms per step).
+    int cn_cap = 0;
+    if (async_compress && attn_ctas > 0 && kvc::kNumSMs - attn_ctas >= (long long)g.Hkv * g.nl)
+      cn_cap = (int)((kvc::kNumSMs - attn_ctas) / ((long long)g.Hkv * g.nl));
     const bool keydiff = cf.policy == KVC_SCORE_KEYDIFF;      // query-agnostic: always scored inside the fused kernel
     const bool fused_score = !keydiff && c->use_tc && g.w * g.G <= kvc::kMaxObsRowsFused;   // few observer rows: likewise
     if (!fused_score && !keydiff) {
@@ -750,10 +761,10 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     {
       ProfScope ps(c, 3, st);
       g.stamps = next_stamp(c, 3);
-      if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, !async_compress, st);
-      else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, !async_compress, st)
-                                         : launch_compress<64, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, !async_compress, st);
-      else e = launch_compress<64, kvc::kScoresGiven>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, !async_compress, st);
+      if (keydiff) e = launch_compress<64, kvc::kScoreKeyDiff>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, !async_compress, cn_cap, st);
+      else if (fused_score) e = D == 128 ? launch_compress<128, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, !async_compress, cn_cap, st)
+                                         : launch_compress<64, kvc::kScoreAttention>(g, dev, tk, tqo, cache, ws, (int)c->elem, pdl, !async_compress, cn_cap, st);
+      else e = launch_compress<64, kvc::kScoresGiven>(g, dev, tk, tk, cache, ws, (int)c->elem, pdl, !async_compress, cn_cap, st);
     }
     if (e != cudaSuccess) return check_cuda(c, e, "compress launch");
     c->launches++;

@@ -427,6 +427,28 @@ def time_steps(fn, steps, barrier):
     return e0.elapsed_time(e1) / 1e3, t0, t1
 
 
+def stamps_as_timed(r: Runner):
+    """Device time stamps of one step in the configuration the benchmark times (compress kernels on the library's
+    side streams when the context has them; calls issued directly, not from the graph): per kernel its launches, mean
+    duration, total and share.  On a side stream a compress kernel gets fewer CTAs per kv-head than in stream order
+    and runs longer, beside the next layer's attention -- this is the table the ncu launch list of the same command
+    compares with."""
+    kv = r.kvc
+    r.step_direct()
+    torch.cuda.synchronize()
+    before = kv.launch_count()
+    r.step_direct()
+    torch.cuda.synchronize()
+    per_step = kv.launch_count() - before
+    kv.profile_device(per_step + 16)
+    r.step_direct()
+    ms, cnt, span_ms = kv.profile_device_read()
+    kv.profile_device(0)
+    tot = sum(ms.values())
+    return {s: dict(launches_per_step=cnt[s], us_per_launch=1e3 * ms[s] / cnt[s], ms_total_per_step=ms[s],
+                    share=ms[s] / tot) for s in ms if cnt[s]} | {"span_ms": span_ms}
+
+
 def profile_pass(r: Runner, steps: int, batched: bool = False, events: bool = False):
     """Per-kernel durations and exact algorithmic work: one call per (block, layer), in stream order, or with
     `batched` one call per block with the layer index in the launch grid.  The durations are device-side time
@@ -628,6 +650,8 @@ def measure(cfg, args, L, local_rank, rank, world, dist, barrier, peaks, steps, 
         if L > 1 and not args.proxy:
             per_b = rates(profile_pass(r, 3, batched=True), peaks)
     out["kernels"], out["kernels_layer_batched"], out["roofline"] = per, per_b, roof
+    if rank == 0 and not args.no_profile and args.mode != "batched" and (flags & 16):
+        out["kernels_as_timed"] = stamps_as_timed(r)
 
     # ---- end to end through the host-buffer entry point
     if primary and not args.no_e2e and not args.proxy:          # (the host-buffer entry point has no proxy variant)
@@ -743,7 +767,7 @@ def main():
             x = measure(c2, args, c2.n_layers, local_rank, rank, world, None, lambda: None, peaks,
                         max(3, min(args.steps, 10)), primary=False)
             extra[name] = {k: x[k] for k in ("value", "ms_per_step", "ms_per_step_in_order", "steps", "launches_per_step",
-                                             "kernel_ms_sum", "kernels", "kernels_layer_batched", "roofline", "roofline_step",
+                                             "kernel_ms_sum", "kernels", "kernels_layer_batched", "kernels_as_timed", "roofline", "roofline_step",
                                              "overlap", "kv_bytes", "clocks", "config") if k in x}
             extra[name]["unit"] = UNIT
 
@@ -754,6 +778,8 @@ def main():
                 "clocks": m["clocks"], "gpu_launches": m["launches_per_step"] * args.steps,
                 "launches_per_step": m["launches_per_step"], "kv_bytes": m["kv_bytes"], "kernels": m["kernels"],
                 "kernels_layer_batched": m["kernels_layer_batched"]}
+        if "kernels_as_timed" in m:
+            line["kernels_as_timed"] = m["kernels_as_timed"]
         for k in ("ms_per_step_in_order", "kernel_ms_sum", "overlap", "roofline_step", "e2e", "cpu_baseline", "output_check"):
             if k in m:
                 line[k] = m[k]

@@ -28,24 +28,30 @@ static constexpr int kStages = 4;                 // K/V ring slots of the atten
 //   warp  9     MMA issuer of tile A, warp 10 of tile B (one lane each).  Per key tile j an issuer
 //               queues O_t += P_t V_j, then S_t = Q_t K_{j+1}^T.  P is handed over in two halves
 //               (64 keys each) so the first PV MMAs start while the second half of the exponentials
-//               is still being computed.
+//               is still being computed.  P -> P V -> next S -> softmax is the row tile's critical chain:
+//               with two row tiles the next S is issued directly behind the second half of P V, and the
+//               commits that free ring slots and publish O follow it.
 //   warp  11    only gives its registers away (setmaxnreg works on groups of four warps)
 // a0: the block's key / value tiles are stored into the cache from their ring slots (TMA stores issued by warp 9).
 // The two softmax groups take turns on the exponentials (named barriers): while one tile's exponentials
 // occupy the CUDA cores the tensor pipe runs the other tile's MMAs; without the hand-over both tiles fall
 // into lockstep and the two pipes idle alternately.  Loading S and finding the maxima is outside the turn.
 // (Measured and dropped: eight softmax warps per row tile, two threads per row, also in the form where a CTA
-// with a single row tile lends it the other tile's warps -- no faster, the per-tile chain is not bound by the
-// instruction count per thread; and a polynomial 2^x on the FMA pipe for part of the columns -- slower.)
+// with a single row tile lends it the other tile's warps -- no faster; a polynomial 2^x on the FMA pipe for part
+// of the columns -- slower; S in two halves of 64 keys with the first issued early -- slower, MMAs with N = 64
+// read Q twice as often; exponentials against the running maximum with the tile's maximum found afterwards --
+// slower, the period is then bound by the two exponential phases, which that form lengthens.)
 // TMEM columns: S_A/P_A [0,128)  S_B/P_B [128,256)  O_A [256,384)  O_B [384,512).
 // The running output is rescaled lazily: a row keeps its reference maximum until the true maximum
 // has grown by more than 2^8, so P stays below 256 and O rarely needs touching.
 //
 // Key split: with cluster size S the CTA of cluster rank s handles key tiles [s*T/S, (s+1)*T/S) of
 // its row-tile pair and ends with a partial (O, m, l).  The partials are exchanged through
-// distributed shared memory: rank s owns rows [s*128/S, (s+1)*128/S) of both tiles, every CTA copies
-// its partial rows (fp32) into the owner's shared memory with remote stores, the cluster
-// synchronises, and each rank combines and writes its rows.  Nothing but the final result goes to HBM.
+// distributed shared memory: rank s owns rows [s*128/S, (s+1)*128/S) of both tiles.  With two row tiles
+// every CTA copies its partial rows (fp32) into the owner's shared memory with remote stores, the cluster
+// synchronises, and each rank combines and writes its rows.  With one row tile the rows (with m and l
+// behind them) leave in one bulk copy per owner, which completes on a barrier of the owner.  Nothing but
+// the final result goes to HBM.
 // Row tiles per CTA: R = 2 as described, or R = 1.  A CTA with one row tile runs it twice over: softmax group and
 // issuer t take its key tiles t, t+2, ... with S, P, O, maximum and row sum of their own (tile B's TMEM columns), and
 // the two partial results are merged at the end.  That costs about 1.1 times as much per row tile and key tile, but

@@ -340,21 +340,22 @@ __global__ void __launch_bounds__(kCompressThreads, 2) compress_kernel(const __g
   // histograms of two consecutive rounds (the second doubles as the list of the last bin's keys): 2 x 8 KB
   int (*hists)[kSelBins] = reinterpret_cast<int (*)[kSelBins]>(smem + kMaxKeysSmem * 8 + 2 * kMaxMovesSmem * 4);
   const bool keys_in_smem = p.n_cand <= kMaxKeysSmem;
-  // One pass builds the keys (four independent loads in flight per thread: the scores come from L2), folds the
+  // One pass builds the keys (twelve independent loads in flight per thread: the scores come from L2), folds the
   // AND and the OR of all keys -- the bits above the highest bit in which any two keys differ are common to all of
   // them (scores of similar magnitude share their exponent bits), and the descent starts below them, so that the
   // first digit already spreads the keys over many bins -- and clears the first histogram.
   unsigned long long k_and = ~0ull, k_or = 0ull;
-  for (int j0 = tid; j0 < p.n_cand; j0 += 4 * kCompressThreads) {
-    float sc[4];
-    int ps[4];
+  constexpr int kKeyLoads = 12;                                  // independent (score, position) loads in flight per thread
+  for (int j0 = tid; j0 < p.n_cand; j0 += kKeyLoads * kCompressThreads) {
+    float sc[kKeyLoads];
+    int ps[kKeyLoads];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kKeyLoads; ++u) {
       const int j = j0 + u * kCompressThreads;
       if (j < p.n_cand) { sc[u] = __ldcg(score + j); ps[u] = pos[j]; }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kKeyLoads; ++u) {
       const int j = j0 + u * kCompressThreads;
       if (j < p.n_cand) {
         const unsigned long long k = select_key(sc[u], ps[u]);

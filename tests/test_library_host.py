@@ -50,6 +50,13 @@ def test_create_validates_configuration():
         assert rc == KVC_EINVAL and not h.value, bad
     assert lib.kvc_create(None, ctypes.byref(ctypes.c_void_p())) == KVC_EINVAL
     assert lib.kvc_destroy(None) == KVC_ESTATE
+    # calls on a dead context are refused before anything touches a device
+    assert lib.kvc_host_flush(None, None) == KVC_ESTATE
+    assert lib.kvc_join(None, None) == KVC_ESTATE
+    # a live context that never used the host entry point has nothing to flush (and needs no device to say so)
+    rc, h = _create()
+    assert rc == KVC_OK and lib.kvc_host_flush(h, None) == KVC_OK
+    assert lib.kvc_destroy(h) == KVC_OK
 
 
 def test_sizes_follow_the_memory_formula():

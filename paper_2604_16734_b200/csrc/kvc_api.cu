@@ -738,8 +738,15 @@ static int run_chunk(kvc_ctx* c, int layer0, int nl, const void* q, long long q_
     // one takes SMs from attention CTAs, which then start late and lengthen the launch everything else waits for
     // (measured on the video workload: 44.3 -> 39.5 ms per step).
     int cn_cap = 0;
-    if (async_compress && attn_ctas > 0 && kvc::kNumSMs - attn_ctas >= (long long)g.Hkv * g.nl)
-      cn_cap = (int)((kvc::kNumSMs - attn_ctas) / ((long long)g.Hkv * g.nl));
+    if (async_compress && attn_ctas > 0 && kvc::kNumSMs - attn_ctas >= (long long)g.Hkv * g.nl) {
+      const long long idle = kvc::kNumSMs - attn_ctas;
+      cn_cap = (int)(idle / ((long long)g.Hkv * g.nl));
+      // ... and a cluster must find its SMs inside one GPC, where the attention leaves about idle / 8 of them: a
+      // cluster larger than that waits for attention CTAs to leave (tiled-image workload, 20 idle SMs, 4 kv-heads:
+      // clusters of 4 or 5 CTAs 2.69e7 tokens/s/layer, of 3 or fewer 2.79e7).
+      const int per_gpc = (int)((idle + 4) / 8);
+      if (cn_cap > per_gpc) cn_cap = per_gpc > 0 ? per_gpc : 1;
+    }
     const bool keydiff = cf.policy == KVC_SCORE_KEYDIFF;      // query-agnostic: always scored inside the fused kernel
     const bool fused_score = !keydiff && c->use_tc && g.w * g.G <= kvc::kMaxObsRowsFused;   // few observer rows: likewise
     if (!fused_score && !keydiff) {
